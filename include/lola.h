@@ -1,0 +1,178 @@
+/*
+ * lola.h - C ABI of the B200 (sm_100a) LoLA per-layer attention step.
+ *
+ * LoLA ("Low-Rank Linear Attention with Sparse Caching", arXiv 2505.23666) keeps every past
+ * key-value pair of an attention head in exactly one of three memories (section "Mitigating Memory
+ * Collisions with Sparse Caching", Fig. 1): a sliding window of the eta most recent pairs, a sparse
+ * global cache G of at most lambda pairs, and the linear-attention state H (D x d_v), s (D) of
+ * Eq. 5.  Pairs leaving the window are scored, together with all of G, by their self-recall error
+ * (Eq. 10) against the current H, s; the lambda highest stay in G (Eq. 12), the rest are folded
+ * into H, s (Eq. 13).  The output (Eq. 14) adds the linear term phi(q)^T H, the sparse-cache term
+ * and the window term over ONE shared denominator.
+ *
+ * Conventions for every entry point
+ *   - All tensors are row-major with the head dimension innermost and contiguous.
+ *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are ordinary
+ *     host memory.  The library never allocates or frees device memory and creates no streams;
+ *     the caller owns every buffer (state, W, q, k, v, out) and must keep W and the state buffer
+ *     alive for the life of the handle.
+ *   - Work is enqueued on the given stream (a cudaStream_t passed as void*; NULL = legacy default
+ *     stream) and the call returns without synchronising unless stated otherwise.  All calls on
+ *     one state must be issued on one stream, or be ordered by the caller.
+ *   - Return value: LOLA_OK (0) or a negative error code.  Argument errors are found on the host
+ *     before anything is enqueued and leave the state untouched.  Nothing throws, prints or exits.
+ *   - One state serves `batch` sequences that advance in lock-step (equal lengths, no padding).
+ *     A "unit" is one (batch row, KV head); the n_q_heads / n_kv_heads query heads of a group share
+ *     their KV head's feature-map weights and its three memories.
+ *   - Token positions are int32 (at most 2^31 - 1 tokens per sequence).
+ */
+#ifndef LOLA_H_
+#define LOLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  LOLA_OK = 0,
+  LOLA_ERR_ARG = -1,         /* null pointer, bad enum, inconsistent view                      */
+  LOLA_ERR_SHAPE = -2,       /* sizes out of range (n_tokens > max_chunk, heads not divisible) */
+  LOLA_ERR_ALIGN = -3,       /* a device pointer is not 16-byte aligned (state: 256-byte)      */
+  LOLA_ERR_SIZE = -4,        /* caller's buffer smaller than lola_state_bytes / staging bytes  */
+  LOLA_ERR_UNSUPPORTED = -5, /* shape outside what the kernels are built for                   */
+  LOLA_ERR_CUDA = -6,        /* a CUDA runtime call or launch failed                           */
+  LOLA_ERR_DEVICE = -7       /* a kernel recorded an internal error in the state's status word */
+};
+
+typedef enum { LOLA_F32 = 0, LOLA_BF16 = 1 } lola_dtype;
+
+/* Feature map phi: R^{d} -> R^{2F}, u = x W.
+ *   LOLA_PHI_SOFTMAX: [softmax(u), softmax(-u)], each over its F entries (the benchmark workloads);
+ *   LOLA_PHI_EXP:     [exp(u), exp(-u)]                                              (Eq. 6).     */
+typedef enum { LOLA_PHI_SOFTMAX = 0, LOLA_PHI_EXP = 1 } lola_phi;
+
+typedef struct lola_config {
+  int32_t batch;         /* B >= 1                                                              */
+  int32_t n_q_heads;     /* Hq, multiple of n_kv_heads                                          */
+  int32_t n_kv_heads;    /* Hkv                                                                 */
+  int32_t head_dim;      /* d = d_k = d_v, 64 or 128                                            */
+  int32_t feat_half;     /* F in [1, 128]; the state has D = 2F feature rows                    */
+  int32_t window;        /* eta >= 0: pairs resident in the sliding window between calls        */
+  int32_t sparse;        /* lambda >= 0: slots of the sparse cache; lambda + max_chunk <= 16384 */
+  int32_t max_chunk;     /* C >= 1: largest n_tokens a prefill call may pass                    */
+  int32_t dtype;         /* lola_dtype of q, k, v, out, W and of the cached keys/values.
+                            H, s, scores and all softmax statistics are always fp32.
+                            LOLA_BF16 additionally rounds phi(K) and H to bf16 inside the Eq. 10
+                            contraction and folds the rounded phi(K) (Eq. 13).                  */
+  int32_t phi_kind;      /* lola_phi                                                            */
+  float softmax_scale;   /* 0 => 1/sqrt(head_dim) (Eq. 2)                                       */
+  uint32_t flags;        /* reserved, must be 0                                                 */
+} lola_config;
+
+/* Opaque host-side handle.  Owns no device memory. */
+typedef struct lola_state lola_state;
+
+/* Host arrays for lola_read_state / lola_write_state.  Every pointer is optional on read (NULL =
+ * skip).  U = batch * n_kv_heads units, unit index = b * n_kv_heads + h.  Elements of *_k / *_v
+ * have the state's dtype (bf16 as raw 16-bit words).                                            */
+typedef struct lola_state_view {
+  float* H;               /* [U, D, d]   Eq. 5 state, fp32                                      */
+  float* s;               /* [U, D]                                                             */
+  int32_t* sparse_count;  /* [U]         occupied slots of G: slots 0 .. count-1                */
+  int32_t* sparse_pos;    /* [U, lambda] token position held by each slot, -1 = empty           */
+  void* sparse_k;         /* [U, lambda, d]                                                     */
+  void* sparse_v;         /* [U, lambda, d]                                                     */
+  float* sparse_score;    /* [U, lambda] self-recall error at the last scored update (NaN: the
+                                         pair has never been scored)                            */
+  float* threshold;       /* [U, 2]      lowest kept / highest folded score of the last scored
+                                         update (NaN before the first one)                      */
+  int32_t* window_count;  /* [U]                                                                */
+  int32_t* window_pos;    /* [U, eta]    position held by ring slot j (= position % eta), -1    */
+  void* window_k;         /* [U, eta, d] ring-slot order                                        */
+  void* window_v;         /* [U, eta, d]                                                        */
+  int64_t* n_seen;        /* [B]         tokens consumed so far                                 */
+  int32_t* status;        /* [1]         sticky device status word, 0 = healthy                 */
+} lola_state_view;
+
+/* Device bytes the caller must provide for one state (a multiple of 256).  0 if cfg is invalid.
+ * Holds H, s, the sparse cache with positions and scores, the window ring, and the small per-unit
+ * work lists the update kernels pass to each other.                                             */
+size_t lola_state_bytes(const lola_config* cfg);
+
+/* Pseudo-code `init`: empty window, empty sparse cache, H = 0, s = 0.
+ *   W_dev     [Hkv, d, F] feature-map weights in cfg->dtype, device, 16-byte aligned; shared by
+ *             queries and keys of the KV head's group.
+ *   state_dev device buffer of at least lola_state_bytes(cfg), 256-byte aligned; zeroed
+ *             asynchronously on `stream`.
+ *   out       receives the handle (host heap; release with lola_destroy_state).
+ * Errors: ARG, SHAPE, ALIGN, SIZE, UNSUPPORTED (device is not compute capability 10.x), CUDA.   */
+int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, size_t state_bytes,
+                    void* stream, lola_state** out);
+
+/* Chunkwise inference (section "Chunkwise Inference", Eq. 15): attend, then evict.
+ * Every query of the chunk sees, with softmax weights, the sparse cache, the resident window and
+ * the chunk itself causally; with linear weights, the H, s of the start of the call (Eq. 14).
+ * Then the chunk joins the window; the pairs that no longer fit (oldest first) are scored together
+ * with all of G by Eq. 10 against the H, s before the fold, the lambda highest errors stay in G
+ * (ties: the older pair stays), and the rest are folded into H, s (Eq. 13).  While fewer than
+ * lambda pairs have ever left the window nothing is scored or folded.
+ *   q   [B, n_tokens, Hq, d] dev      k, v [B, n_tokens, Hkv, d] dev      out [B, n_tokens, Hq, d] dev
+ *   out may be NULL: only the caches advance (q is then ignored and may be NULL).
+ *   1 <= n_tokens <= max_chunk.
+ * Errors: ARG, SHAPE, ALIGN, CUDA.                                                              */
+int lola_prefill_chunk(lola_state* st, const void* q, const void* k, const void* v, int32_t n_tokens,
+                       void* out, void* stream);
+
+/* Generation step (Eq. 11-14): update, then attend.  The new pair enters the window; if the window
+ * overflows its oldest pair is evicted, E = G u {evicted} is scored against the current H, s, the
+ * lowest-error pair of E is folded and the others form G; then Eq. 14 is evaluated over the updated
+ * G, H, s and the window including the new pair.
+ *   q [B, Hq, d] dev      k, v [B, Hkv, d] dev      out [B, Hq, d] dev (required)
+ * Errors: ARG, ALIGN, CUDA.                                                                     */
+int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v, void* out, void* stream);
+
+/* Same two operations for callers whose tensors live in HOST memory.  `staging_dev` is a device
+ * buffer of at least lola_staging_bytes(cfg, n_tokens) bytes (256-byte aligned) that the call uses
+ * for the device copies of q, k, v and out; inputs are copied in, the step runs, out is copied back
+ * and the stream is synchronised before returning, so out_host is valid on return.  Pinned host
+ * memory makes the copies asynchronous with respect to the host but is not required.
+ * Errors: as above plus SIZE.                                                                   */
+size_t lola_staging_bytes(const lola_config* cfg, int32_t n_tokens);
+int lola_prefill_chunk_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host,
+                            int32_t n_tokens, void* out_host, void* staging_dev, size_t staging_bytes,
+                            void* stream);
+int lola_decode_step_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host,
+                          void* out_host, void* staging_dev, size_t staging_bytes, void* stream);
+
+/* Copies the three memories to the host arrays of `view` and synchronises `stream`.  The paper has
+ * no counterpart; this is how results are inspected and checkpointed.  Returns LOLA_ERR_DEVICE if
+ * the sticky status word is non-zero (the arrays are still filled).                             */
+int lola_read_state(const lola_state* st, const lola_state_view* view, void* stream);
+
+/* Replaces the three memories by the host arrays of `view` (all of H, s, sparse_count, sparse_pos,
+ * sparse_k, sparse_v, window_count, window_pos, window_k, window_v, n_seen are required;
+ * sparse_score and threshold are optional).  Window rows may be given in any order: row j of a unit
+ * holds position window_pos[j] and is stored at ring slot position % eta.  The view must describe a
+ * reachable state: all n_seen equal, window = the last min(eta, n_seen) positions, sparse_count =
+ * min(lambda, n_seen - window_count) for every unit; otherwise LOLA_ERR_ARG.  Synchronises.     */
+int lola_write_state(lola_state* st, const lola_state_view* view, void* stream);
+
+/* Number of kernel launches this handle has enqueued so far. */
+int64_t lola_launch_count(const lola_state* st);
+
+/* Tokens consumed so far per sequence. */
+int64_t lola_tokens_seen(const lola_state* st);
+
+/* Releases the host handle only; device buffers stay with the caller. */
+int lola_destroy_state(lola_state* st);
+
+/* Static description of an error code. */
+const char* lola_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOLA_H_ */

@@ -138,6 +138,8 @@ class UnitState:
         self.last_kept_min = np.nan                        # lowest kept / highest folded score
         self.last_folded_max = np.nan                      # at the most recent scored update
         self.n_scored_updates = 0
+        self.last_E_pos = np.zeros((0,), dtype=np.int64)   # eligible set and its scores at the most
+        self.last_E_score = np.zeros((0,))                 # recent scored update (for tie-aware checks)
 
     # -- helpers
     def _rq(self, x: np.ndarray) -> np.ndarray:
@@ -173,6 +175,7 @@ class UnitState:
             self.last_kept_min = float(score[keep].min())
             self.last_folded_max = float(score[lose].max())
             self.n_scored_updates += 1
+            self.last_E_pos, self.last_E_score = E_pos.copy(), score.copy()
         # Eq. 13: H += sum phi(k) v^T, s += sum phi(k) over the pairs that are not kept
         self.H = self.H + f[lose].T @ E_v[lose]
         self.s = self.s + f[lose].sum(axis=0)

@@ -1,0 +1,430 @@
+// Host side of the C ABI declared in include/lola.h: argument checks, the carve-up of the caller's
+// state buffer, the per-call geometry (every count is a function of the tokens seen so far, so no
+// device value is ever read back to decide a launch), and the launches themselves.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/lola.h"
+#include "lola_generic.cuh"
+#include "lola_params.h"
+
+using namespace lola;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct StateLayout {
+  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, total;
+};
+
+bool config_ok(const lola_config* c) {
+  if (!c) return false;
+  if (c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->feat_half < 1 || c->feat_half > 128) return false;
+  if (c->window < 0 || c->sparse < 0 || c->max_chunk < 1) return false;
+  if ((int64_t)c->sparse + c->max_chunk > 16384) return false;
+  if (c->dtype != LOLA_F32 && c->dtype != LOLA_BF16) return false;
+  if (c->phi_kind != LOLA_PHI_SOFTMAX && c->phi_kind != LOLA_PHI_EXP) return false;
+  if (!(c->softmax_scale >= 0.f) || c->flags != 0) return false;
+  if ((int64_t)2 * c->feat_half * c->head_dim > (int64_t)kUpdThreads * kUpdEPT) return false;
+  return true;
+}
+
+StateLayout make_layout(const lola_config& c) {
+  const size_t U = (size_t)c.batch * c.n_kv_heads, d = c.head_dim, D = 2 * (size_t)c.feat_half;
+  const size_t es = c.dtype == LOLA_BF16 ? 2 : 4;
+  const size_t lam = c.sparse, eta = c.window, cm = c.max_chunk;
+  StateLayout l{};
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  l.status = take(256);
+  l.H = take(U * D * d * 4);
+  l.s = take(U * D * 4);
+  l.gk = take(U * lam * d * es);
+  l.gv = take(U * lam * d * es);
+  l.gpos = take(U * lam * 4);
+  l.score = take(U * (lam + cm) * 4);
+  l.wk = take(U * eta * d * es);
+  l.wv = take(U * eta * d * es);
+  l.fold_idx = take(U * cm * 4);
+  l.move_src = take(U * cm * 4);
+  l.move_dst = take(U * cm * 4);
+  l.counts = take(U * 4 * 4);
+  l.thr = take(U * 2 * 4);
+  l.total = o;
+  return l;
+}
+
+inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+struct Geometry {
+  int cw, r, r_pos0, count_g, mode, new_count_g;
+};
+
+// Counts before/after consuming n tokens when n_seen tokens have been consumed already.
+Geometry plan(const lola_config& c, int64_t n_seen, int n) {
+  Geometry g{};
+  g.cw = (int)std::min<int64_t>(c.window, n_seen);
+  g.r = std::max(0, g.cw + n - c.window);
+  g.r_pos0 = (int)(n_seen - g.cw);
+  g.count_g = (int)std::min<int64_t>(c.sparse, n_seen - g.cw);
+  const int nE = g.count_g + g.r;
+  if (g.r == 0) g.mode = UPD_NONE;
+  else if (c.sparse == 0) g.mode = UPD_FOLD_ALL;
+  else if (nE <= c.sparse) g.mode = UPD_APPEND;
+  else g.mode = UPD_SELECT;
+  g.new_count_g = std::min(c.sparse, nE);
+  return g;
+}
+
+template <typename T, int DPL>
+int set_smem_attrs(int D) {
+  cudaError_t e;
+  e = cudaFuncSetAttribute(k_attend<T, DPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(attend_smem_floats<DPL>(D) * 4));
+  if (e != cudaSuccess) return LOLA_ERR_CUDA;
+  e = cudaFuncSetAttribute(k_score<T, DPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(score_smem_floats<DPL>(D) * 4));
+  if (e != cudaSuccess) return LOLA_ERR_CUDA;
+  e = cudaFuncSetAttribute(k_update<T, DPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(update_smem_floats<DPL>(D) * 4));
+  if (e != cudaSuccess) return LOLA_ERR_CUDA;
+  return LOLA_OK;
+}
+
+}  // namespace
+
+struct lola_state {
+  lola_config cfg;
+  Layer L;
+  StateLayout lay;
+  char* base;
+  int64_t n_seen;
+  int64_t launches;
+};
+
+namespace {
+
+template <typename T, int DPL>
+int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
+  const Layer& L = st->L;
+  dim3 grid((L.g * c.nq + kAttRows - 1) / kAttRows, L.B * L.Hkv);
+  k_attend<T, DPL><<<grid, 256, attend_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+  st->launches++;
+  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
+template <typename T, int DPL>
+int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
+  const Layer& L = st->L;
+  const int U = L.B * L.Hkv;
+  if (c.mode == UPD_SELECT) {
+    const int nE = c.count_g + c.r;
+    dim3 grid((nE + kScoreRows - 1) / kScoreRows, U);
+    k_score<T, DPL><<<grid, 256, score_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+    st->launches++;
+    if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
+  }
+  if (c.mode != UPD_NONE) {
+    const int nE = c.count_g + c.r;
+    size_t sm = (c.mode == UPD_SELECT) ? ((size_t)nE * 8 + (size_t)L.cmax * 4 + (size_t)nE + 16) : 0;
+    k_select<<<U, 256, sm, s>>>(L, c);
+    st->launches++;
+    if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
+  }
+  k_update<T, DPL><<<U, kUpdThreads, update_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+  st->launches++;
+  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
+template <typename T, int DPL>
+int run_prefill(lola_state* st, Call c, cudaStream_t s) {
+  int rc = LOLA_OK;
+  if (c.out) rc = launch_attend<T, DPL>(st, c, s);
+  if (rc != LOLA_OK) return rc;
+  return launch_update_chain<T, DPL>(st, c, s);
+}
+
+template <typename T, int DPL>
+int run_decode(lola_state* st, Call c, cudaStream_t s) {
+  int rc = launch_update_chain<T, DPL>(st, c, s);
+  if (rc != LOLA_OK) return rc;
+  return launch_attend<T, DPL>(st, c, s);
+}
+
+#define LOLA_DISPATCH(fn, st, ...)                                                            \
+  ((st)->cfg.dtype == LOLA_BF16                                                               \
+       ? ((st)->cfg.head_dim == 128 ? fn<__nv_bfloat16, 4>(st, __VA_ARGS__) : fn<__nv_bfloat16, 2>(st, __VA_ARGS__)) \
+       : ((st)->cfg.head_dim == 128 ? fn<float, 4>(st, __VA_ARGS__) : fn<float, 2>(st, __VA_ARGS__)))
+
+size_t elem_size(const lola_config& c) { return c.dtype == LOLA_BF16 ? 2 : 4; }
+
+}  // namespace
+
+extern "C" {
+
+size_t lola_state_bytes(const lola_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return make_layout(*cfg).total;
+}
+
+int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, size_t state_bytes, void* stream,
+                    lola_state** out) {
+  if (!cfg || !W_dev || !state_dev || !out) return LOLA_ERR_ARG;
+  if (!config_ok(cfg)) {
+    if (cfg->head_dim != 64 && cfg->head_dim != 128 && cfg->head_dim > 0) return LOLA_ERR_UNSUPPORTED;
+    return LOLA_ERR_SHAPE;
+  }
+  if (!aligned(W_dev, 16) || !aligned(state_dev, kAlign)) return LOLA_ERR_ALIGN;
+  StateLayout lay = make_layout(*cfg);
+  if (state_bytes < lay.total) return LOLA_ERR_SIZE;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (prop.major != 10) return LOLA_ERR_UNSUPPORTED;
+
+  lola_state* st = new (std::nothrow) lola_state();
+  if (!st) return LOLA_ERR_ARG;
+  st->cfg = *cfg;
+  st->lay = lay;
+  st->base = (char*)state_dev;
+  st->n_seen = 0;
+  st->launches = 0;
+  Layer& L = st->L;
+  L.B = cfg->batch; L.Hq = cfg->n_q_heads; L.Hkv = cfg->n_kv_heads; L.g = cfg->n_q_heads / cfg->n_kv_heads;
+  L.d = cfg->head_dim; L.F = cfg->feat_half; L.D = 2 * cfg->feat_half;
+  L.eta = cfg->window; L.lam = cfg->sparse; L.cmax = cfg->max_chunk;
+  L.phi_kind = cfg->phi_kind; L.bf16 = cfg->dtype == LOLA_BF16;
+  L.scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  char* b = st->base;
+  L.status = (int*)(b + lay.status);
+  L.H = (float*)(b + lay.H); L.s = (float*)(b + lay.s);
+  L.gk = b + lay.gk; L.gv = b + lay.gv; L.gpos = (int*)(b + lay.gpos); L.score = (float*)(b + lay.score);
+  L.wk = b + lay.wk; L.wv = b + lay.wv;
+  L.fold_idx = (int*)(b + lay.fold_idx); L.move_src = (int*)(b + lay.move_src); L.move_dst = (int*)(b + lay.move_dst);
+  L.counts = (int*)(b + lay.counts); L.thr = (float*)(b + lay.thr);
+  L.W = W_dev;
+
+  int rc = LOLA_OK;
+  if (cfg->dtype == LOLA_BF16) rc = cfg->head_dim == 128 ? set_smem_attrs<__nv_bfloat16, 4>(L.D) : set_smem_attrs<__nv_bfloat16, 2>(L.D);
+  else rc = cfg->head_dim == 128 ? set_smem_attrs<float, 4>(L.D) : set_smem_attrs<float, 2>(L.D);
+  if (rc == LOLA_OK && cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 9 * 16384 + 4 * 16384 + 64) != cudaSuccess)
+    rc = LOLA_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (rc == LOLA_OK && cudaMemsetAsync(b, 0, lay.total, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
+  const size_t U = (size_t)cfg->batch * cfg->n_kv_heads;
+  // positions -1, scores and thresholds NaN (all-ones bit pattern)
+  if (rc == LOLA_OK && cfg->sparse > 0 && cudaMemsetAsync(L.gpos, 0xFF, U * cfg->sparse * 4, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
+  if (rc == LOLA_OK && cudaMemsetAsync(L.score, 0xFF, U * ((size_t)cfg->sparse + cfg->max_chunk) * 4, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
+  if (rc == LOLA_OK && cudaMemsetAsync(L.thr, 0xFF, U * 2 * 4, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
+  if (rc != LOLA_OK) { delete st; return rc; }
+  *out = st;
+  return LOLA_OK;
+}
+
+int lola_prefill_chunk(lola_state* st, const void* q, const void* k, const void* v, int32_t n_tokens, void* out,
+                       void* stream) {
+  if (!st || !k || !v) return LOLA_ERR_ARG;
+  if (out && !q) return LOLA_ERR_ARG;
+  if (n_tokens < 1 || n_tokens > st->cfg.max_chunk) return LOLA_ERR_SHAPE;
+  if (st->n_seen + n_tokens > 0x7fffffffLL) return LOLA_ERR_SHAPE;
+  if (!aligned(k, 16) || !aligned(v, 16) || (out && (!aligned(q, 16) || !aligned(out, 16)))) return LOLA_ERR_ALIGN;
+  const Geometry g = plan(st->cfg, st->n_seen, n_tokens);
+  Call c{};
+  c.q = q; c.k = k; c.v = v; c.out = out;
+  c.n = n_tokens; c.nq = n_tokens; c.n_seen = (int)st->n_seen;
+  c.r = g.r; c.r_pos0 = g.r_pos0; c.count_g = g.count_g; c.mode = g.mode;
+  c.att_g = g.count_g; c.att_w0 = (int)st->n_seen - g.cw; c.att_wn = g.cw; c.att_chunk = n_tokens;
+  int rc = LOLA_DISPATCH(run_prefill, st, c, (cudaStream_t)stream);
+  if (rc == LOLA_OK) st->n_seen += n_tokens;
+  return rc;
+}
+
+int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v, void* out, void* stream) {
+  if (!st || !q || !k || !v || !out) return LOLA_ERR_ARG;
+  if (st->n_seen + 1 > 0x7fffffffLL) return LOLA_ERR_SHAPE;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16)) return LOLA_ERR_ALIGN;
+  const Geometry g = plan(st->cfg, st->n_seen, 1);
+  Call c{};
+  c.q = q; c.k = k; c.v = v; c.out = out;
+  c.n = 1; c.nq = 1; c.n_seen = (int)st->n_seen;
+  c.r = g.r; c.r_pos0 = g.r_pos0; c.count_g = g.count_g; c.mode = g.mode;
+  const int cw_after = (int)std::min<int64_t>(st->cfg.window, st->n_seen + 1);
+  c.att_g = g.new_count_g; c.att_w0 = (int)(st->n_seen + 1) - cw_after; c.att_wn = cw_after; c.att_chunk = 0;
+  int rc = LOLA_DISPATCH(run_decode, st, c, (cudaStream_t)stream);
+  if (rc == LOLA_OK) st->n_seen += 1;
+  return rc;
+}
+
+size_t lola_staging_bytes(const lola_config* cfg, int32_t n_tokens) {
+  if (!config_ok(cfg) || n_tokens < 1) return 0;
+  const size_t es = elem_size(*cfg), d = cfg->head_dim, B = cfg->batch;
+  const size_t qb = align_up(B * n_tokens * cfg->n_q_heads * d * es);
+  const size_t kb = align_up(B * n_tokens * cfg->n_kv_heads * d * es);
+  return 2 * qb + 2 * kb;
+}
+
+static int run_host(lola_state* st, const void* qh, const void* kh, const void* vh, int32_t n, void* oh, void* stg,
+                    size_t stg_bytes, void* stream, bool decode) {
+  if (!st || !kh || !vh || !stg) return LOLA_ERR_ARG;
+  if ((decode || oh) && !qh) return LOLA_ERR_ARG;
+  if (decode && !oh) return LOLA_ERR_ARG;
+  if (n < 1 || n > st->cfg.max_chunk) return LOLA_ERR_SHAPE;
+  if (!aligned(stg, kAlign)) return LOLA_ERR_ALIGN;
+  if (stg_bytes < lola_staging_bytes(&st->cfg, n)) return LOLA_ERR_SIZE;
+  const lola_config& c = st->cfg;
+  const size_t es = elem_size(c), d = c.head_dim, B = c.batch;
+  const size_t qbytes = B * n * c.n_q_heads * d * es, kbytes = B * n * c.n_kv_heads * d * es;
+  const size_t qb = align_up(qbytes), kb = align_up(kbytes);
+  char* p = (char*)stg;
+  void *qd = p, *kd = p + qb, *vd = p + qb + kb, *od = p + qb + 2 * kb;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (oh && cudaMemcpyAsync(qd, qh, qbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (cudaMemcpyAsync(kd, kh, kbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (cudaMemcpyAsync(vd, vh, kbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  int rc = decode ? lola_decode_step(st, qd, kd, vd, od, stream)
+                  : lola_prefill_chunk(st, oh ? qd : nullptr, kd, vd, n, oh ? od : nullptr, stream);
+  if (rc != LOLA_OK) return rc;
+  if (oh && cudaMemcpyAsync(oh, od, qbytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return LOLA_ERR_CUDA;
+  return LOLA_OK;
+}
+
+int lola_prefill_chunk_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host,
+                            int32_t n_tokens, void* out_host, void* staging_dev, size_t staging_bytes, void* stream) {
+  return run_host(st, q_host, k_host, v_host, n_tokens, out_host, staging_dev, staging_bytes, stream, false);
+}
+
+int lola_decode_step_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host, void* out_host,
+                          void* staging_dev, size_t staging_bytes, void* stream) {
+  return run_host(st, q_host, k_host, v_host, 1, out_host, staging_dev, staging_bytes, stream, true);
+}
+
+int lola_read_state(const lola_state* st, const lola_state_view* view, void* stream) {
+  if (!st || !view) return LOLA_ERR_ARG;
+  const lola_config& c = st->cfg;
+  const Layer& L = st->L;
+  const size_t U = (size_t)c.batch * c.n_kv_heads, d = c.head_dim, D = L.D, es = elem_size(c);
+  const size_t lam = c.sparse, eta = c.window, cm = c.max_chunk;
+  cudaStream_t s = (cudaStream_t)stream;
+  auto d2h = [&](void* dst, const void* src, size_t bytes) {
+    if (!dst || bytes == 0) return true;
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  };
+  bool ok = true;
+  ok = ok && d2h(view->H, L.H, U * D * d * 4);
+  ok = ok && d2h(view->s, L.s, U * D * 4);
+  ok = ok && d2h(view->sparse_pos, L.gpos, U * lam * 4);
+  ok = ok && d2h(view->sparse_k, L.gk, U * lam * d * es);
+  ok = ok && d2h(view->sparse_v, L.gv, U * lam * d * es);
+  ok = ok && d2h(view->window_k, L.wk, U * eta * d * es);
+  ok = ok && d2h(view->window_v, L.wv, U * eta * d * es);
+  ok = ok && d2h(view->threshold, L.thr, U * 2 * 4);
+  int status = 0;
+  ok = ok && d2h(&status, L.status, 4);
+  if (view->sparse_score && lam > 0) {   // the first lambda entries of each unit's score row
+    ok = ok && cudaMemcpy2DAsync(view->sparse_score, lam * 4, L.score, (lam + cm) * 4, lam * 4, U,
+                                 cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  }
+  if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return LOLA_ERR_CUDA;
+  const Geometry g = plan(c, st->n_seen, 0);
+  for (size_t u = 0; u < U; ++u) {
+    if (view->sparse_count) view->sparse_count[u] = g.count_g;
+    if (view->window_count) view->window_count[u] = g.cw;
+    if (view->window_pos) {
+      for (size_t j = 0; j < eta; ++j) view->window_pos[u * eta + j] = -1;
+      for (int64_t p = st->n_seen - g.cw; p < st->n_seen; ++p) view->window_pos[u * eta + (size_t)(p % (int64_t)eta)] = (int32_t)p;
+    }
+  }
+  if (view->n_seen) for (int b = 0; b < c.batch; ++b) view->n_seen[b] = st->n_seen;
+  if (view->status) view->status[0] = status;
+  return status == 0 ? LOLA_OK : LOLA_ERR_DEVICE;
+}
+
+int lola_write_state(lola_state* st, const lola_state_view* v, void* stream) {
+  if (!st || !v) return LOLA_ERR_ARG;
+  if (!v->H || !v->s || !v->sparse_count || !v->window_count || !v->n_seen) return LOLA_ERR_ARG;
+  const lola_config& c = st->cfg;
+  const Layer& L = st->L;
+  const size_t U = (size_t)c.batch * c.n_kv_heads, d = c.head_dim, D = L.D, es = elem_size(c);
+  const size_t lam = c.sparse, eta = c.window, cm = c.max_chunk;
+  if (lam > 0 && (!v->sparse_pos || !v->sparse_k || !v->sparse_v)) return LOLA_ERR_ARG;
+  if (eta > 0 && (!v->window_pos || !v->window_k || !v->window_v)) return LOLA_ERR_ARG;
+  const int64_t n_seen = v->n_seen[0];
+  if (n_seen < 0 || n_seen > 0x7fffffffLL) return LOLA_ERR_ARG;
+  for (int b = 0; b < c.batch; ++b) if (v->n_seen[b] != n_seen) return LOLA_ERR_ARG;
+  const Geometry g = plan(c, n_seen, 0);
+  for (size_t u = 0; u < U; ++u) {
+    if (v->sparse_count[u] != g.count_g || v->window_count[u] != g.cw) return LOLA_ERR_ARG;
+  }
+  // window rows to ring order
+  std::vector<char> wk(U * eta * d * es, 0), wv(U * eta * d * es, 0);
+  for (size_t u = 0; u < U && eta > 0; ++u) {
+    std::vector<char> seen(eta, 0);
+    for (int j = 0; j < g.cw; ++j) {
+      int64_t p = v->window_pos[u * eta + j];
+      if (p < n_seen - g.cw || p >= n_seen) return LOLA_ERR_ARG;
+      size_t slot = (size_t)(p % (int64_t)eta);
+      if (seen[slot]) return LOLA_ERR_ARG;
+      seen[slot] = 1;
+      std::memcpy(&wk[(u * eta + slot) * d * es], (const char*)v->window_k + (u * eta + j) * d * es, d * es);
+      std::memcpy(&wv[(u * eta + slot) * d * es], (const char*)v->window_v + (u * eta + j) * d * es, d * es);
+    }
+  }
+  std::vector<float> sc(U * (lam + cm));
+  { uint32_t nanbits = 0xFFFFFFFFu; float nanv; std::memcpy(&nanv, &nanbits, 4); std::fill(sc.begin(), sc.end(), nanv); }
+  if (v->sparse_score)
+    for (size_t u = 0; u < U; ++u) std::memcpy(&sc[u * (lam + cm)], v->sparse_score + u * lam, lam * 4);
+  cudaStream_t s = (cudaStream_t)stream;
+  auto h2d = [&](void* dst, const void* src, size_t bytes) {
+    if (bytes == 0) return true;
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  };
+  bool ok = true;
+  ok = ok && h2d(L.H, v->H, U * D * d * 4);
+  ok = ok && h2d(L.s, v->s, U * D * 4);
+  ok = ok && h2d(L.gpos, v->sparse_pos, U * lam * 4);
+  ok = ok && h2d(L.gk, v->sparse_k, U * lam * d * es);
+  ok = ok && h2d(L.gv, v->sparse_v, U * lam * d * es);
+  ok = ok && h2d(L.score, sc.data(), sc.size() * 4);
+  ok = ok && h2d(L.wk, wk.data(), wk.size());
+  ok = ok && h2d(L.wv, wv.data(), wv.size());
+  if (v->threshold) ok = ok && h2d(L.thr, v->threshold, U * 2 * 4);
+  if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return LOLA_ERR_CUDA;   // host staging dies here
+  st->n_seen = n_seen;
+  return LOLA_OK;
+}
+
+int64_t lola_launch_count(const lola_state* st) { return st ? st->launches : -1; }
+int64_t lola_tokens_seen(const lola_state* st) { return st ? st->n_seen : -1; }
+
+int lola_destroy_state(lola_state* st) {
+  if (!st) return LOLA_ERR_ARG;
+  delete st;
+  return LOLA_OK;
+}
+
+const char* lola_strerror(int code) {
+  switch (code) {
+    case LOLA_OK: return "ok";
+    case LOLA_ERR_ARG: return "invalid argument (null pointer, bad enum or inconsistent state view)";
+    case LOLA_ERR_SHAPE: return "size out of range";
+    case LOLA_ERR_ALIGN: return "pointer not sufficiently aligned";
+    case LOLA_ERR_SIZE: return "caller-provided buffer too small";
+    case LOLA_ERR_UNSUPPORTED: return "shape or device not supported by this build (needs sm_100)";
+    case LOLA_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
+    case LOLA_ERR_DEVICE: return "a kernel recorded an internal error in the state's status word";
+    default: return "unknown error code";
+  }
+}
+
+}  // extern "C"

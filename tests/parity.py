@@ -1,0 +1,158 @@
+"""Lock-step comparison of the CUDA library with the CPU oracle on the same seeded inputs.
+
+Both sides consume the same arrays call by call.  After every call the outputs are compared
+element by element and the three memories are compared: sparse-cache membership must be identical
+except where the oracle's own scores show a near-tie at the selection threshold; then the library's
+state is replaced by the oracle's (oracle -> GPU, never the other way) and the run continues, and the
+number of such events is reported.
+
+Tolerances (stated by the workload's contract):
+  fp32 mode: |gpu - ref| <= 1e-4 * (|ref| + mean|ref|) for outputs, H and s; membership exact except
+             pairs whose oracle score lies within 1e-5 * max(1, |tau|) of the threshold tau.
+  bf16 mode: |gpu - ref| <= 2e-2 for outputs and H (s: 2e-2 relative to its scale); near-tie band
+             2^-8 * max(1, |tau|): one bf16 unit in the last place of a rounded phi(k) or H entry moves
+             a score by at most that much.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle.lola_oracle import LolaOracle, config_for
+from paper_2505_23666_b200 import binding
+from paper_2505_23666_b200.workloads import Workload, WorkloadInputs
+
+
+def tolerances(dtype: str):
+    if dtype == "bf16":
+        return dict(kind="abs", out=2e-2, H=2e-2, tie=2.0 ** -8)
+    return dict(kind="rel", out=1e-4, H=1e-4, tie=1e-5)
+
+
+def close(gpu: np.ndarray, ref: np.ndarray, tol: float, kind: str):
+    """Returns (ok, worst ratio of error to allowance)."""
+    gpu = np.asarray(gpu, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    err = np.abs(gpu - ref)
+    if kind == "rel":
+        allow = tol * (np.abs(ref) + np.abs(ref).mean() + 1e-30)
+    else:
+        allow = np.full_like(err, tol)
+    ratio = float((err / allow).max()) if err.size else 0.0
+    return bool(np.isfinite(gpu).all() and ratio <= 1.0), ratio
+
+
+class Lockstep:
+    def __init__(self, wl: Workload, rows=None, threads: int = 8, device="cuda:0", inputs: WorkloadInputs = None):
+        self.wl = wl
+        self.rows = list(range(wl.batch)) if rows is None else list(rows)
+        self.inputs = inputs or WorkloadInputs(wl)
+        B = len(self.rows)
+        self.tol = tolerances(wl.dtype)
+        self.ocfg = config_for(wl, batch=B)
+        self.oracle = LolaOracle(self.ocfg, self.inputs.W.astype(np.float64), threads=threads)
+        self.cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window,
+                                       wl.sparse, max(wl.chunk, 1), dtype=wl.dtype)
+        self.layer = binding.LolaLayer(self.cfg, self.inputs.W, device=device)
+        self.resyncs = 0
+        self.scored_updates = 0
+        self.worst = {"out": 0.0, "H": 0.0, "s": 0.0, "score": 0.0}
+        self.calls = 0
+
+    # ------------------------------------------------------------------ steps
+    def prefill(self, t0: int, n: int, want_out: bool = True, check_state: bool = True):
+        q, k, v = self.inputs.prefill_tokens(t0, n, batch_rows=self.rows, need_q=want_out)
+        L = self.layer
+        dq = L.to_device(q) if want_out else None
+        out = L.prefill_chunk(dq, L.to_device(k), L.to_device(v), want_out=want_out)
+        ref = self.oracle.prefill_chunk(q, k, v, want_out=want_out)
+        if want_out:
+            self._cmp_out(out.float().cpu().numpy(), ref, f"prefill t0={t0}")
+        self.calls += 1
+        if check_state:
+            self.check_state(f"prefill t0={t0}")
+
+    def decode(self, step: int, check_state: bool = True):
+        q, k, v = self.inputs.decode_token(step, batch_rows=self.rows)
+        L = self.layer
+        out = L.decode_step(L.to_device(q), L.to_device(k), L.to_device(v))
+        ref = self.oracle.decode_step(q, k, v)
+        self._cmp_out(out.float().cpu().numpy(), ref, f"decode step={step}")
+        self.calls += 1
+        if check_state:
+            self.check_state(f"decode step={step}")
+
+    # ------------------------------------------------------------------ comparisons
+    def _cmp_out(self, gpu, ref, where):
+        ok, ratio = close(gpu, ref, self.tol["out"], self.tol["kind"])
+        self.worst["out"] = max(self.worst["out"], ratio)
+        assert ok, f"{where}: output outside tolerance (worst error/allowance {ratio:.3g})"
+
+    def check_state(self, where: str = ""):
+        g = self.layer.read_state()
+        o = self.oracle.read_state()
+        assert int(g["status"][0]) == 0, f"{where}: device status {int(g['status'][0])}"
+        assert np.array_equal(g["n_seen"], o["n_seen"]), where
+        assert np.array_equal(g["sparse_count"], o["sparse_count"]), f"{where}: sparse counts differ"
+        assert np.array_equal(g["window_count"], o["window_count"]), f"{where}: window counts differ"
+        B, Hk = g["sparse_count"].shape
+        need_resync = False
+        for b in range(B):
+            for h in range(Hk):
+                u = self.oracle.units[b][h]
+                m, w = int(o["sparse_count"][b, h]), int(o["window_count"][b, h])
+                # window: same positions, exact copies of the pairs
+                gp = g["window_pos"][b, h]
+                sel = gp >= 0
+                order = np.argsort(gp[sel])
+                assert np.array_equal(gp[sel][order], o["window_pos"][b, h, :w]), f"{where}: window positions"
+                assert np.array_equal(g["window_k"][b, h][sel][order], o["window_k"][b, h, :w].astype(np.float32)), where
+                assert np.array_equal(g["window_v"][b, h][sel][order], o["window_v"][b, h, :w].astype(np.float32)), where
+                # sparse cache membership
+                gpos = g["sparse_pos"][b, h, :m].astype(np.int64)
+                assert np.all(g["sparse_pos"][b, h, m:] == -1), f"{where}: stale slots"
+                assert len(set(gpos.tolist())) == m, f"{where}: duplicate members"
+                so = np.argsort(gpos)
+                if np.array_equal(gpos[so], o["sparse_pos"][b, h, :m]):
+                    assert np.array_equal(g["sparse_k"][b, h, :m][so], o["sparse_k"][b, h, :m].astype(np.float32)), where
+                    assert np.array_equal(g["sparse_v"][b, h, :m][so], o["sparse_v"][b, h, :m].astype(np.float32)), where
+                    for name in ("H", "s"):
+                        tol = self.tol["H"]
+                        if name == "s" and self.tol["kind"] == "abs":
+                            tol = self.tol["H"] * max(1.0, float(np.abs(o["s"][b, h]).max()))
+                        ok, ratio = close(g[name][b, h], o[name][b, h], tol, self.tol["kind"])
+                        self.worst[name] = max(self.worst[name], ratio)
+                        assert ok, f"{where}: {name} of unit ({b},{h}) outside tolerance ({ratio:.3g})"
+                    # scores of the members, where both sides have scored them
+                    gs, os_ = g["sparse_score"][b, h, :m][so], o["sparse_score"][b, h, :m]
+                    both = ~np.isnan(os_)
+                    assert np.array_equal(np.isnan(gs), np.isnan(os_)), f"{where}: scored/unscored flags"
+                    if both.any():
+                        stol = 1e-4 if self.tol["kind"] == "rel" else 2.0 ** -8
+                        ratio = float((np.abs(gs[both] - os_[both]) / (stol * np.maximum(1.0, np.abs(os_[both])))).max())
+                        self.worst["score"] = max(self.worst["score"], ratio)
+                        assert ratio <= 1.0, f"{where}: member scores differ ({ratio:.3g})"
+                else:
+                    self._assert_near_tie(u, set(gpos.tolist()), where, (b, h))
+                    need_resync = True
+        self.scored_updates = sum(u.n_scored_updates for row in self.oracle.units for u in row)
+        if need_resync:
+            self.resyncs += 1
+            self.layer.write_state(o)
+
+    def _assert_near_tie(self, u, gpu_members: set, where, unit):
+        """Membership differs: every pair on the wrong side must be a near-tie in the ORACLE's scores of
+        this update, and the difference must be a swap of equal numbers of pairs."""
+        orc_members = set(int(p) for p in u.G_pos)
+        only_g, only_o = gpu_members - orc_members, orc_members - gpu_members
+        assert len(only_g) == len(only_o) > 0, f"{where} unit {unit}: membership sizes differ"
+        sc = {int(p): float(s) for p, s in zip(u.last_E_pos, u.last_E_score)}
+        tau = 0.5 * (u.last_kept_min + u.last_folded_max)
+        band = self.tol["tie"] * max(1.0, abs(tau))
+        for p in sorted(only_g | only_o):
+            assert p in sc, f"{where} unit {unit}: pair {p} was not eligible in this update"
+            assert abs(sc[p] - tau) <= band, \
+                f"{where} unit {unit}: pair {p} differs and is no near-tie (score {sc[p]:.9g}, threshold {tau:.9g})"
+
+    def summary(self):
+        return dict(calls=self.calls, resyncs=self.resyncs, scored_updates=self.scored_updates, worst=dict(self.worst))

@@ -1,0 +1,149 @@
+"""CUDA library vs CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_23666_b200.workloads import WORKLOADS, WorkloadInputs, small_case
+from tests.parity import Lockstep
+
+pytestmark = pytest.mark.gpu
+
+
+def drive(ls: Lockstep, tokens: int, chunk: int, decode_steps: int = 0, want_out=True):
+    t = 0
+    while t < tokens:
+        n = min(chunk, tokens - t)
+        ls.prefill(t, n, want_out=want_out)
+        t += n
+    for sidx in range(decode_steps):
+        ls.decode(sidx)
+    return ls.summary()
+
+
+# ---- small cases: several tiles, ragged tails, every update mode, both dtypes, both head sizes
+SMALL = [
+    # name                d    F   eta lam  C   tokens decode dtype
+    ("f32_d64",          64,  64,  32, 48,  32, 300,   12,   "f32"),
+    ("f32_d128",        128,  64,  16, 40,  16, 200,   10,   "f32"),
+    ("f32_ragged",       64,  64,  24, 37,  20, 211,    9,   "f32"),   # C != eta, odd sizes, partial last chunk
+    ("f32_chunk_gt_win", 64,  64,   8, 20,  32, 160,    6,   "f32"),   # chunk larger than the window
+    ("f32_no_window",    64,  64,   0, 16,  16,  96,   20,   "f32"),   # eta = 0
+    ("f32_no_sparse",    64,  64,  16,  0,  16,  96,   20,   "f32"),   # lambda = 0: window + linear attention
+    ("f32_linear_only",  64,  64,   0,  0,  16,  64,   20,   "f32"),   # decode = causal linear attention
+    ("f32_all_softmax",  64,  64,  16, 512, 16, 128,   20,   "f32"),   # caches never fill: H stays 0
+    ("f32_F32",          64,  32,  16, 24,  16, 128,    8,   "f32"),   # D = 64
+    ("f32_F128",         64, 128,  16, 24,  16, 128,    8,   "f32"),   # D = 256
+    ("bf16_d64",         64,  64,  32, 48,  32, 300,   12,   "bf16"),
+    ("bf16_d128",       128,  64,  16, 40,  16, 200,   10,   "bf16"),
+    ("bf16_ragged",     128,  64,  24, 37,  20, 211,    9,   "bf16"),
+    ("bf16_lam1",       128,  64,  16,  1,  16, 128,   10,   "bf16"),
+]
+
+
+@pytest.mark.parametrize("name,d,F,eta,lam,C,tokens,decode,dtype", SMALL, ids=[s[0] for s in SMALL])
+def test_small_cases(name, d, F, eta, lam, C, tokens, decode, dtype):
+    wl = small_case(name, batch=2, n_q_heads=4, n_kv_heads=2, head_dim=d, feat_half=F, tokens=tokens, chunk=C,
+                    window=eta, sparse=lam, dtype=dtype, seed=11, decode_steps=decode,
+                    scale_a=(0.125 if dtype == "f32" else 1.0))
+    ls = Lockstep(wl, threads=1)
+    summ = drive(ls, tokens, C, decode)
+    assert summ["resyncs"] <= max(1, summ["scored_updates"] // 50), summ
+    if name == "f32_all_softmax":
+        st = ls.layer.read_state()
+        assert np.all(st["H"] == 0) and np.all(st["s"] == 0)
+
+
+def test_exp_feature_map():
+    wl = small_case("exp", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
+                    dtype="f32", seed=5, decode_steps=8, scale_a=0.125)
+    from oracle.lola_oracle import config_for, LolaOracle
+    from paper_2505_23666_b200 import binding
+    ls = Lockstep(wl, threads=1)
+    # rebuild both sides with the Eq. 6 feature map
+    ls.ocfg = config_for(wl, phi_kind="exp")
+    ls.oracle = LolaOracle(ls.ocfg, ls.inputs.W.astype(np.float64))
+    ls.cfg = binding.make_config(1, 2, 2, 64, 64, 16, 24, 16, dtype="f32", phi_kind="exp")
+    ls.layer = binding.LolaLayer(ls.cfg, ls.inputs.W)
+    drive(ls, 160, 16, 8)
+
+
+def test_state_only_prefill_and_host_entry_points():
+    """out = NULL advances the caches exactly like a call with outputs; the host-buffer entry points
+    give the same results as the device ones."""
+    wl = small_case("host", batch=2, n_q_heads=4, n_kv_heads=2, tokens=192, chunk=32, window=32, sparse=40,
+                    dtype="bf16", seed=3, decode_steps=4)
+    a, b = Lockstep(wl, threads=1), Lockstep(wl, threads=1)
+    for t in range(0, 192, 32):
+        a.prefill(t, 32, want_out=False)
+        q, k, v = b.inputs.prefill_tokens(t, 32)
+        tq, tk, tv = (torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in (q, k, v))
+        out = torch.empty_like(tq).pin_memory()
+        b.layer.prefill_chunk_host(tq, tk, tv, out)
+        ref = b.oracle.prefill_chunk(q, k, v)
+        b._cmp_out(out.float().numpy(), ref, f"host prefill {t}")
+        b.check_state("host prefill")
+    sa, sb = a.layer.read_state(), b.layer.read_state()
+    for key in ("H", "s", "sparse_pos", "sparse_k", "window_k"):
+        assert np.array_equal(sa[key], sb[key]), key
+    q, k, v = b.inputs.decode_token(0)
+    tq, tk, tv = (torch.from_numpy(x).to(torch.bfloat16) for x in (q, k, v))
+    out = torch.empty_like(tq)
+    b.layer.decode_step_host(tq, tk, tv, out)
+    b._cmp_out(out.float().numpy(), b.oracle.decode_step(q, k, v), "host decode")
+
+
+def test_write_state_round_trip():
+    wl = small_case("rt", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
+                    dtype="f32", seed=9, scale_a=0.125)
+    ls = Lockstep(wl, threads=1)
+    drive(ls, 96, 16)
+    ls.layer.write_state(ls.oracle.read_state())      # import the oracle's state, then keep going
+    ls.check_state("after import")
+    for t in range(96, 160, 16):
+        ls.prefill(t, 16)
+
+
+def test_argument_errors_leave_state_untouched():
+    from paper_2505_23666_b200 import binding as b
+    wl = small_case("err", batch=1, n_q_heads=2, n_kv_heads=2, tokens=64, chunk=16, window=16, sparse=8, dtype="f32")
+    ls = Lockstep(wl, threads=1)
+    L = ls.layer
+    q, k, v = ls.inputs.prefill_tokens(0, 32)
+    dq, dk, dv = L.to_device(q), L.to_device(k), L.to_device(v)
+    out = torch.empty_like(dq)
+    s = torch.cuda.current_stream().cuda_stream
+    assert b.lola_prefill_chunk(L.handle, dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), 32, out.data_ptr(), s) == b.LOLA_ERR_SHAPE
+    assert b.lola_prefill_chunk(L.handle, dq.data_ptr(), 0, dv.data_ptr(), 16, out.data_ptr(), s) == b.LOLA_ERR_ARG
+    assert b.lola_prefill_chunk(L.handle, dq.data_ptr() + 4, dk.data_ptr(), dv.data_ptr(), 16, out.data_ptr(), s) == b.LOLA_ERR_ALIGN
+    assert b.lola_decode_step(L.handle, dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), 0, s) == b.LOLA_ERR_ARG
+    assert L.tokens_seen == 0
+    bad = b.make_config(1, 3, 2, 64, 64, 16, 8, 16)
+    assert b.lola_state_bytes(bad) == 0
+    with pytest.raises(b.LolaError):
+        b.LolaLayer(b.make_config(1, 2, 2, 96, 64, 16, 8, 16), np.zeros((2, 96, 64), np.float32))
+    ls.prefill(0, 16)                                   # the state still works
+
+
+# ---- the five workloads
+def test_cfg0_full():
+    wl = WORKLOADS["cfg0"]
+    ls = Lockstep(wl)
+    summ = drive(ls, wl.tokens, wl.chunk)
+    print("cfg0", summ)
+    assert summ["resyncs"] == 0 or summ["resyncs"] <= 1
+
+
+def test_cfg1_full():
+    wl = WORKLOADS["cfg1"]
+    ls = Lockstep(wl)
+    summ = drive(ls, wl.tokens, wl.chunk)
+    print("cfg1", summ)
+    assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100)
+
+
+def test_cfg2_full():
+    wl = WORKLOADS["cfg2"]
+    ls = Lockstep(wl)
+    summ = drive(ls, wl.tokens, wl.chunk)
+    print("cfg2", summ)
+    assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100)
