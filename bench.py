@@ -1,0 +1,528 @@
+#!/usr/bin/env python
+"""Benchmark of the LoLA per-layer attention step on B200 (one process per GPU).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg0|cfg1|cfg4] [--impl reference]
+
+One "step" is one pass of the whole hot path over the workload's batch:
+  * prefill workloads (cfg0, cfg1, cfg2, cfg4): reset the state, then the full prefill in chunks of C tokens
+    through lola_prefill_chunk (attention, self-recall error, selection, fold, window roll);
+  * decode workload (cfg3): all `decode_steps` single-token lola_decode_step calls on a state built (untimed)
+    by the seeded prefill; the state is restored from a device copy before every step.
+The printed value is tokens/s per layer (whole job, all GPUs).  The default line is the 8B-shaped prefill
+(cfg2) and carries the decode workload (cfg3) as a second entry under "decode".
+
+Units are independent, so N GPUs each run the same per-GPU workload on their own batch rows (weak scaling,
+no data-path collective); torch.distributed is used only for the barrier and the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "LoLA tokens/s per layer"
+UNIT = "tokens/s"
+
+
+# ----------------------------------------------------------------------------- algorithmic work
+def geometry(wl, n_seen, n):
+    cw = min(wl.window, n_seen)
+    r = max(0, cw + n - wl.window)
+    count_g = min(wl.sparse, n_seen - cw)
+    nE = count_g + r
+    scored = r > 0 and wl.sparse > 0 and nE > wl.sparse
+    nfold = (nE - wl.sparse) if scored else (r if wl.sparse == 0 else 0)
+    return cw, r, count_g, nE, scored, nfold
+
+
+def prefill_call_flops(wl, n_seen, n):
+    """Algorithmic FLOPs of one lola_prefill_chunk call per unit, split by step of the method."""
+    g, d, F, D = wl.group, wl.head_dim, wl.feat_half, wl.feat_dim
+    cw, r, count_g, nE, scored, nfold = geometry(wl, n_seen, n)
+    rows = g * n
+    keys = count_g + cw + (n + 1) / 2.0                       # causal half of the chunk
+    attend = 2 * 2 * rows * keys * d + 2 * rows * d * F + 2 * rows * D * d + 2 * rows * D
+    score = (2 * nE * d * F + 2 * nE * D * d + 2 * nE * D) if scored else 0
+    update = (2 * nfold * d * F + 2 * nfold * D * d) if nfold else 0
+    return {"attend": attend, "score": score, "select": 0.0, "update": update}
+
+
+def decode_step_bytes(wl, n_seen):
+    """Algorithmic HBM bytes of one decode step per unit: every resident array read once, the changed
+    parts written once."""
+    g, d, D = wl.group, wl.head_dim, wl.feat_dim
+    es = 2 if wl.dtype == "bf16" else 4
+    cw, r, count_g, nE, scored, nfold = geometry(wl, n_seen, 1)
+    rd = 2 * count_g * d * es + 4 * count_g + 2 * min(wl.window, n_seen + 1) * d * es + D * d * 4 + D * 4 + (g + 2) * d * es
+    wr = (D * d * 4 + D * 4 if nfold else 0) + g * d * es + 2 * d * es + (2 * d * es if r else 0)
+    return rd + wr
+
+
+def decode_step_flops(wl, n_seen):
+    g, d, F, D = wl.group, wl.head_dim, wl.feat_half, wl.feat_dim
+    cw, r, count_g, nE, scored, nfold = geometry(wl, n_seen, 1)
+    keys = min(wl.sparse, nE) + min(wl.window, n_seen + 1)
+    fl = 2 * 2 * g * keys * d + 2 * g * d * F + 2 * g * D * d
+    if scored:
+        fl += 2 * nE * d * F + 2 * nE * D * d + 2 * nE * D
+    fl += nfold * (2 * d * F + 2 * D * d)
+    return fl
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0, t1):
+        rows = [s for (t, s) in self.samples if t0 <= t <= t1] or [s for (_, s) in self.samples]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in rows:
+            f = [x.strip() for x in row.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except Exception:
+                continue
+            for nme, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- helpers
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def rank_rows(rank: int, per_rank_batch: int):
+    """Global batch rows owned by a rank: rank r runs rows [r*B, (r+1)*B) of the seeded generator."""
+    return list(range(rank * per_rank_batch, (rank + 1) * per_rank_batch))
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def oracle_prefill_sample(wl, inputs, rows, tokens, threads):
+    """Times the CPU oracle as it stands on `rows` x `tokens` of the workload. Returns (tokens/s, seconds)."""
+    from oracle.lola_oracle import LolaOracle, config_for
+    orc = LolaOracle(config_for(wl, batch=len(rows)), inputs.W.astype(np.float64), threads=threads)
+    chunks = [inputs.prefill_tokens(t, min(wl.chunk, tokens - t), batch_rows=rows) for t in range(0, tokens, wl.chunk)]
+    t0 = time.time()
+    for q, k, v in chunks:
+        orc.prefill_chunk(q, k, v)
+    dt = time.time() - t0
+    return len(rows) * tokens / dt, dt
+
+
+def oracle_decode_sample(wl, inputs, rows, prefill_tokens, steps, threads):
+    from oracle.lola_oracle import LolaOracle, config_for
+    orc = LolaOracle(config_for(wl, batch=len(rows)), inputs.W.astype(np.float64), threads=threads)
+    for t in range(0, prefill_tokens, wl.chunk):
+        _, k, v = inputs.prefill_tokens(t, wl.chunk, batch_rows=rows, need_q=False)
+        orc.prefill_chunk(None, k, v, want_out=False)
+    toks = [inputs.decode_token(i, batch_rows=rows) for i in range(steps)]
+    t0 = time.time()
+    for q, k, v in toks:
+        orc.decode_step(q, k, v)
+    dt = time.time() - t0
+    return len(rows) * steps / dt, dt
+
+
+# ----------------------------------------------------------------------------- prefill workloads
+def bench_prefill(wl, args, rank, local_rank, world, peaks):
+    import torch
+    from paper_2505_23666_b200 import binding
+    from paper_2505_23666_b200.workloads import WorkloadInputs
+    dev = torch.device(f"cuda:{local_rank}")
+    inputs = WorkloadInputs(wl.with_(batch=wl.batch * world))
+    rows = rank_rows(rank, wl.batch)
+    B, T, C = wl.batch, wl.tokens, wl.chunk
+    nch = T // C
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    # host arrays in call order: [chunk, B, C, heads, d]
+    hq = torch.empty((nch, B, C, wl.n_q_heads, wl.head_dim), dtype=tdt).pin_memory()
+    hk = torch.empty((nch, B, C, wl.n_kv_heads, wl.head_dim), dtype=tdt).pin_memory()
+    hv = torch.empty_like(hk).pin_memory()
+    blk = 64                                                      # chunks generated per generator call
+    for c0 in range(0, nch, blk):
+        c1 = min(nch, c0 + blk)
+        q, k, v = inputs.prefill_tokens(c0 * C, (c1 - c0) * C, batch_rows=rows)
+        for src, dst in ((q, hq), (k, hk), (v, hv)):
+            a = torch.from_numpy(src).reshape(B, c1 - c0, C, src.shape[2], src.shape[3]).permute(1, 0, 2, 3, 4)
+            dst[c0:c1].copy_(a)
+    dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
+    dout = torch.empty_like(dq)
+    hout = torch.empty_like(hq).pin_memory()
+    cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window, wl.sparse, C,
+                              dtype=wl.dtype)
+    layer = binding.LolaLayer(cfg, inputs.W, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        layer.reset()
+        for c in range(nch):
+            layer.prefill_chunk(dq[c], dk[c], dv[c], out=dout[c])
+
+    def step_host():
+        layer.reset()
+        for c in range(nch):
+            layer.prefill_chunk_host(hq[c], hk[c], hv[c], hout[c])
+
+    sampler = ClockSampler(local_rank)
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize(dev)
+    barrier(world)
+    l0 = layer.launches
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    w1 = time.time()
+    barrier(world)
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    launches = layer.launches - l0
+    clocks = sampler.summary(w0, w1)
+
+    # end to end through the host-buffer entry point (copies inside the timed region)
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    step_host()
+    torch.cuda.synchronize(dev)
+    barrier(world)
+    t0 = time.time()
+    for _ in range(e2e_steps):
+        step_host()
+    torch.cuda.synchronize(dev)
+    e2e_ms = max_over_ranks((time.time() - t0) * 1e3, world, dev)
+    sampler.stop()
+
+    # per-kernel device times (events around every launch), separate pass so the headline is unperturbed
+    layer.profile(True)
+    prof_steps = max(1, min(3, args.steps))
+    for _ in range(prof_steps):
+        step()
+    kms, kn = layer.profile_read()
+    layer.profile(False)
+    flops = {k: 0.0 for k in ("attend", "score", "select", "update")}
+    for c in range(nch):
+        for k, f in prefill_call_flops(wl, c * C, C).items():
+            flops[k] += f * wl.units
+    total_flops = sum(flops.values())
+    dom = max(kms, key=kms.get)
+    dom_launch_ms = kms[dom] / kn[dom]
+    dom_flops_per_launch = flops[dom] * prof_steps / kn[dom]
+    peak = peaks["bf16_tflops_sustained"]
+    achieved = dom_flops_per_launch / (dom_launch_ms * 1e-3) / 1e12
+    tokens_per_step = B * T
+    res = {
+        "metric": METRIC, "value": world * tokens_per_step * args.steps / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": f"{wl.name}: prefill B={B} x {T} tokens, chunk {C}, window {wl.window}, "
+                               f"lambda {wl.sparse}, Hq {wl.n_q_heads}, Hkv {wl.n_kv_heads}, d {wl.head_dim}",
+                   "l2": "inputs (q,k,v,out %.0f MB) larger than L2; state %.1f MB resident" %
+                         ((dq.numel() * 2 + dk.numel() * 2) * dq.element_size() / 1e6, layer.nbytes / 1e6),
+                   "per_chunk_call_us": ms / args.steps / nch * 1e3},
+        "clocks": clocks,
+        "e2e": {"value": world * tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": (hq.numel() + 2 * hk.numel()) * hq.element_size(),
+                "d2h_bytes_per_step": hout.numel() * hout.element_size(), "steps": e2e_steps},
+        "gpu_launches": launches,
+        "roofline": {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                     "launch_us": dom_launch_ms * 1e3,
+                     "whole_step": {"achieved": total_flops / (ms / args.steps * 1e-3) / 1e12,
+                                    "frac": total_flops / (ms / args.steps * 1e-3) / 1e12 / peak},
+                     "kernel_ms_per_step": {k: v / prof_steps for k, v in kms.items()},
+                     "kernel_launches_per_step": {k: v / prof_steps for k, v in kn.items()}},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        ncores = len(os.sched_getaffinity(0))
+        srows = rows[:min(len(rows), 2)]
+        stoks = min(T, 4096)
+        v, dt = oracle_prefill_sample(wl, inputs, srows, stoks, ncores)
+        res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ncores, "kind": "oracle",
+                               "sample": f"batch rows {srows}, first {stoks} tokens ({dt:.1f} s)"}
+    layer.close()
+    return res
+
+
+# ----------------------------------------------------------------------------- decode workload
+def bench_decode(wl, args, rank, local_rank, world, peaks):
+    import torch
+    from paper_2505_23666_b200 import binding
+    from paper_2505_23666_b200.workloads import WorkloadInputs
+    dev = torch.device(f"cuda:{local_rank}")
+    inputs = WorkloadInputs(wl.with_(batch=wl.batch * world))
+    rows = rank_rows(rank, wl.batch)
+    B, C, S = wl.batch, wl.chunk, wl.decode_steps
+    T = args.decode_prefill if args.decode_prefill else wl.tokens
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window, wl.sparse, C,
+                              dtype=wl.dtype)
+    layer = binding.LolaLayer(cfg, inputs.W, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    # untimed: build the state with the seeded prefill (keys and values only)
+    blk = 8
+    for c0 in range(0, T // C, blk):
+        c1 = min(T // C, c0 + blk)
+        _, k, v = inputs.prefill_tokens(c0 * C, (c1 - c0) * C, batch_rows=rows, need_q=False)
+        tk = torch.from_numpy(k).to(dev, tdt).reshape(B, c1 - c0, C, wl.n_kv_heads, wl.head_dim)
+        tv = torch.from_numpy(v).to(dev, tdt).reshape(B, c1 - c0, C, wl.n_kv_heads, wl.head_dim)
+        for c in range(c1 - c0):
+            layer.prefill_chunk(None, tk[:, c].contiguous(), tv[:, c].contiguous(), want_out=False)
+    torch.cuda.synchronize(dev)
+    snapshot = layer.state.clone()
+    toks = [inputs.decode_token(i, batch_rows=rows) for i in range(S)]
+    hq = torch.stack([torch.from_numpy(t[0]) for t in toks]).to(tdt).pin_memory()
+    hk = torch.stack([torch.from_numpy(t[1]) for t in toks]).to(tdt).pin_memory()
+    hv = torch.stack([torch.from_numpy(t[2]) for t in toks]).to(tdt).pin_memory()
+    dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
+    dout = torch.empty_like(dq)
+    hout = torch.empty_like(hq).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def restore():
+        layer.state.copy_(snapshot)
+        binding.lola_set_tokens_seen(layer.handle, T)
+
+    def step():
+        for i in range(S):
+            layer.decode_step(dq[i], dk[i], dv[i], out=dout[i])
+
+    def step_host():
+        for i in range(S):
+            layer.decode_step_host(hq[i], hk[i], hv[i], hout[i])
+
+    sampler = ClockSampler(local_rank)
+    for _ in range(args.warmup):
+        restore()
+        step()
+    torch.cuda.synchronize(dev)
+    barrier(world)
+    l0 = layer.launches
+    total_ms = 0.0
+    w0 = time.time()
+    for _ in range(args.steps):
+        restore()
+        flush.fill_(1)                                            # L2 flush between timed steps
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        total_ms += e0.elapsed_time(e1)
+    w1 = time.time()
+    barrier(world)
+    ms = max_over_ranks(total_ms, world, dev)
+    launches = layer.launches - l0
+    clocks = sampler.summary(w0, w1)
+
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    restore()
+    step_host()
+    e2e_total = 0.0
+    for _ in range(e2e_steps):
+        restore()
+        torch.cuda.synchronize(dev)
+        t0 = time.time()
+        step_host()
+        torch.cuda.synchronize(dev)
+        e2e_total += (time.time() - t0) * 1e3
+    e2e_ms = max_over_ranks(e2e_total, world, dev)
+    sampler.stop()
+
+    layer.profile(True)
+    restore()
+    step()
+    kms, kn = layer.profile_read()
+    layer.profile(False)
+    step_bytes = sum(decode_step_bytes(wl, T + i) for i in range(S)) * wl.units / S    # per decode call
+    step_flops = sum(decode_step_flops(wl, T + i) for i in range(S)) * wl.units / S
+    call_ms = ms / args.steps / S
+    kernel_ms_per_call = sum(kms.values()) / S
+    peak = peaks["hbm_gbs"]
+    achieved = step_bytes / (kernel_ms_per_call * 1e-3) / 1e9
+    res = {
+        "metric": METRIC, "value": world * B * S * args.steps / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": f"{wl.name}: decode B={B}, {S} single-token calls after a {T}-token prefill, "
+                               f"window {wl.window}, lambda {wl.sparse}, Hq {wl.n_q_heads}, Hkv {wl.n_kv_heads}, "
+                               f"d {wl.head_dim}",
+                   "l2": "state %.0f MB larger than L2; L2 flushed between timed steps" % (layer.nbytes / 1e6),
+                   "per_decode_call_us": call_ms * 1e3},
+        "clocks": clocks,
+        "e2e": {"value": world * B * S * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": (hq.numel() + 2 * hk.numel()) * hq.element_size(),
+                "d2h_bytes_per_step": hout.numel() * hout.element_size(), "steps": e2e_steps},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "+".join(sorted(kms)) + " (all kernels of one decode call)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "peak_source": peaks["source"], "bytes_per_call": step_bytes, "flops_per_call": step_flops,
+                     "launch_us": kernel_ms_per_call * 1e3,
+                     "kernel_us_per_call": {k: v / S * 1e3 for k, v in kms.items()}},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        ncores = len(os.sched_getaffinity(0))
+        stoks, ssteps = 2048, 32
+        v, dt = oracle_decode_sample(wl, inputs, rows[:1], stoks, ssteps, ncores)
+        res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ncores, "kind": "oracle",
+                               "sample": f"batch row {rows[0]}, {ssteps} decode steps after a {stoks}-token prefill "
+                                         f"(caches full; {dt:.1f} s timed)"}
+    layer.close()
+    return res
+
+
+# ----------------------------------------------------------------------------- reference arm (the oracle)
+def bench_reference(wl, args):
+    from paper_2505_23666_b200.workloads import WorkloadInputs
+    inputs = WorkloadInputs(wl)
+    ncores = len(os.sched_getaffinity(0))
+    if wl.decode_steps:
+        sample = "batch row 0, 32 decode steps after a 2048-token prefill per step"
+        fn = lambda: oracle_decode_sample(wl, inputs, [0], 2048, 32, ncores)   # noqa: E731
+        per_step = 32
+    else:
+        stoks = min(wl.tokens, 4096)
+        sample = f"batch row 0, first {stoks} tokens per step"
+        fn = lambda: oracle_prefill_sample(wl, inputs, [0], stoks, ncores)      # noqa: E731
+        per_step = stoks
+    for _ in range(args.warmup):
+        fn()
+    tot = 0.0
+    for _ in range(args.steps):
+        _, dt = fn()
+        tot += dt
+    value = per_step * args.steps / tot
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{wl.name} (CPU oracle on a bounded sample: {sample})"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": ncores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="default", choices=["default", "cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--decode-prefill", type=int, default=0, help="tokens of the untimed prefill of cfg3 (0 = full)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="default line without the cfg3 entry")
+    args = ap.parse_args()
+    from paper_2505_23666_b200.workloads import WORKLOADS
+    rank, local_rank, world = dist_env()
+    main_name = "cfg2" if args.workload == "default" else args.workload
+    wl = WORKLOADS[main_name]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        args.warmup = min(args.warmup, 1)
+        args.steps = args.steps or 3
+        print(json.dumps(bench_reference(wl, args)), flush=True)
+        return
+
+    import torch
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    from paper_2505_23666_b200 import build as _b
+    if rank == 0:
+        _b.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+        dist.barrier()
+    peaks = load_peaks()
+    default_steps = {"cfg0": 20, "cfg1": 20, "cfg2": 10, "cfg3": 5, "cfg4": 3}
+    user_steps = args.steps
+    args.steps = user_steps or default_steps[main_name]
+    res = (bench_decode if wl.decode_steps else bench_prefill)(wl, args, rank, local_rank, world, peaks)
+    if args.workload == "default" and not args.no_decode:
+        wl3 = WORKLOADS["cfg3"]
+        a3 = argparse.Namespace(**vars(args))
+        a3.steps = user_steps or default_steps["cfg3"]
+        r3 = bench_decode(wl3, a3, rank, local_rank, world, peaks)
+        res["decode"] = {k: r3[k] for k in ("value", "unit", "ms_per_step", "steps", "config", "e2e", "gpu_launches",
+                                             "roofline", "clocks") if k in r3}
+        if "cpu_baseline" in r3:
+            res["decode"]["cpu_baseline"] = r3["cpu_baseline"]
+    if rank == 0:
+        print(json.dumps(res), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -112,6 +112,9 @@ size_t lola_state_bytes(const lola_config* cfg);
 int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, size_t state_bytes,
                     void* stream, lola_state** out);
 
+/* Back to the state lola_init_state leaves (pseudo-code `init`), asynchronously on `stream`. */
+int lola_reset_state(lola_state* st, void* stream);
+
 /* Chunkwise inference (section "Chunkwise Inference", Eq. 15): attend, then evict.
  * Every query of the chunk sees, with softmax weights, the sparse cache, the resident window and
  * the chunk itself causally; with linear weights, the H, s of the start of the call (Eq. 14).
@@ -160,11 +163,31 @@ int lola_read_state(const lola_state* st, const lola_state_view* view, void* str
  * min(lambda, n_seen - window_count) for every unit; otherwise LOLA_ERR_ARG.  Synchronises.     */
 int lola_write_state(lola_state* st, const lola_state_view* view, void* stream);
 
+/* Per-kernel device timing (no counterpart in the paper; used by the benchmark's roofline figures).
+ * While enabled, every kernel launch of this handle is bracketed by a pair of CUDA events on the
+ * call's stream.  lola_profile_read synchronises `stream`, writes the accumulated milliseconds and
+ * launch counts per kernel kind since the last read (arrays of LOLA_N_KERNEL_KINDS) and clears them. */
+enum {
+  LOLA_KERNEL_ATTEND = 0,  /* Eq. 14: softmax over sparse cache + window + chunk, linear term         */
+  LOLA_KERNEL_SCORE = 1,   /* Eq. 10: self-recall error of the eligible set                         */
+  LOLA_KERNEL_SELECT = 2,  /* Eq. 12: top-lambda                                                    */
+  LOLA_KERNEL_UPDATE = 3,  /* Eq. 13 fold, moves into the sparse cache, window roll                 */
+  LOLA_KERNEL_DECODE = 4,  /* fused generation step                                                 */
+  LOLA_N_KERNEL_KINDS = 8
+};
+int lola_profile_enable(lola_state* st, int enable);
+int lola_profile_read(lola_state* st, double* ms_by_kind, int64_t* launches_by_kind, void* stream);
+
 /* Number of kernel launches this handle has enqueued so far. */
 int64_t lola_launch_count(const lola_state* st);
 
 /* Tokens consumed so far per sequence. */
 int64_t lola_tokens_seen(const lola_state* st);
+
+/* For callers that restore the state buffer themselves (a device-to-device copy of a snapshot taken
+ * after n_seen tokens): tells the handle how many tokens that buffer has consumed.  Every count the
+ * library uses (window fill, occupied slots) follows from this number.                          */
+int lola_set_tokens_seen(lola_state* st, int64_t n_seen);
 
 /* Releases the host handle only; device buffers stay with the caller. */
 int lola_destroy_state(lola_state* st);

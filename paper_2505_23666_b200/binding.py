@@ -61,8 +61,12 @@ def _load() -> C.CDLL:
         "lola_decode_step_host": (C.c_int, [vp, vp, vp, vp, vp, vp, sz, vp]),
         "lola_read_state": (C.c_int, [vp, viewp, vp]),
         "lola_write_state": (C.c_int, [vp, viewp, vp]),
+        "lola_reset_state": (C.c_int, [vp, vp]),
+        "lola_profile_enable": (C.c_int, [vp, C.c_int]),
+        "lola_profile_read": (C.c_int, [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), vp]),
         "lola_launch_count": (i64, [vp]),
         "lola_tokens_seen": (i64, [vp]),
+        "lola_set_tokens_seen": (C.c_int, [vp, i64]),
         "lola_destroy_state": (C.c_int, [vp]),
         "lola_strerror": (C.c_char_p, [C.c_int]),
     }
@@ -75,7 +79,7 @@ def _load() -> C.CDLL:
 _lib = _load()
 EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_decode_step", "lola_staging_bytes",
            "lola_prefill_chunk_host", "lola_decode_step_host", "lola_read_state", "lola_write_state",
-           "lola_launch_count", "lola_tokens_seen", "lola_destroy_state", "lola_strerror"]
+           "lola_reset_state", "lola_profile_enable", "lola_profile_read", "lola_launch_count", "lola_tokens_seen", "lola_set_tokens_seen", "lola_destroy_state", "lola_strerror"]
 
 
 # ---- one-to-one wrappers (pointers are integers: tensor.data_ptr(), stream.cuda_stream) ----
@@ -125,12 +129,37 @@ def lola_write_state(st: int, view: lola_state_view, stream: int) -> int:
     return _lib.lola_write_state(st, C.byref(view), stream)
 
 
+def lola_reset_state(st: int, stream: int) -> int:
+    return _lib.lola_reset_state(st, stream)
+
+
+KERNEL_KINDS = ["attend", "score", "select", "update", "decode", "kind5", "kind6", "kind7"]
+
+
+def lola_profile_enable(st: int, enable: bool) -> int:
+    return _lib.lola_profile_enable(st, 1 if enable else 0)
+
+
+def lola_profile_read(st: int, stream: int):
+    """Returns ({kind: ms}, {kind: launches}) accumulated since the last read."""
+    ms = (C.c_double * 8)()
+    n = (C.c_int64 * 8)()
+    rc = _lib.lola_profile_read(st, ms, n, stream)
+    if rc != LOLA_OK:
+        raise LolaError(rc, "lola_profile_read")
+    return ({k: ms[i] for i, k in enumerate(KERNEL_KINDS) if n[i]}, {k: n[i] for i, k in enumerate(KERNEL_KINDS) if n[i]})
+
+
 def lola_launch_count(st: int) -> int:
     return int(_lib.lola_launch_count(st))
 
 
 def lola_tokens_seen(st: int) -> int:
     return int(_lib.lola_tokens_seen(st))
+
+
+def lola_set_tokens_seen(st: int, n_seen: int) -> int:
+    return _lib.lola_set_tokens_seen(st, int(n_seen))
 
 
 def lola_destroy_state(st: int) -> int:
@@ -277,6 +306,15 @@ class LolaLayer:
             keep[k] = a
         view = lola_state_view(**{k: (v.data_ptr() if v.numel() else None) for k, v in keep.items()})
         _check(lola_write_state(self.handle, view, self._stream()), "lola_write_state")
+
+    def reset(self):
+        _check(lola_reset_state(self.handle, self._stream()), "lola_reset_state")
+
+    def profile(self, enable: bool):
+        _check(lola_profile_enable(self.handle, enable), "lola_profile_enable")
+
+    def profile_read(self):
+        return lola_profile_read(self.handle, self._stream())
 
     @property
     def launches(self) -> int:

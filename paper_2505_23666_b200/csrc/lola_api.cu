@@ -103,6 +103,8 @@ int set_smem_attrs(int D) {
 
 }  // namespace
 
+struct ProfRecord { int kind; cudaEvent_t a, b; };
+
 struct lola_state {
   lola_config cfg;
   Layer L;
@@ -110,16 +112,37 @@ struct lola_state {
   char* base;
   int64_t n_seen;
   int64_t launches;
+  bool profiling = false;
+  std::vector<ProfRecord> records;     // events in use since the last lola_profile_read
+  std::vector<ProfRecord> pool;        // events ready for reuse
 };
 
 namespace {
+
+// Brackets one launch with a pair of events when profiling is on (kind = LOLA_KERNEL_*).
+struct LaunchScope {
+  lola_state* st; cudaStream_t s; ProfRecord rec; bool on;
+  LaunchScope(lola_state* st_, int kind, cudaStream_t s_) : st(st_), s(s_), on(st_->profiling) {
+    st->launches++;
+    if (!on) return;
+    if (!st->pool.empty()) { rec = st->pool.back(); st->pool.pop_back(); }
+    else if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) { on = false; return; }
+    rec.kind = kind;
+    cudaEventRecord(rec.a, s);
+  }
+  ~LaunchScope() {
+    if (!on) return;
+    cudaEventRecord(rec.b, s);
+    st->records.push_back(rec);
+  }
+};
 
 template <typename T, int DPL>
 int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   dim3 grid((L.g * c.nq + kAttRows - 1) / kAttRows, L.B * L.Hkv);
+  LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
   k_attend<T, DPL><<<grid, 256, attend_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
-  st->launches++;
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
@@ -130,19 +153,19 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   if (c.mode == UPD_SELECT) {
     const int nE = c.count_g + c.r;
     dim3 grid((nE + kScoreRows - 1) / kScoreRows, U);
+    LaunchScope scope(st, LOLA_KERNEL_SCORE, s);
     k_score<T, DPL><<<grid, 256, score_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
-    st->launches++;
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   }
   if (c.mode != UPD_NONE) {
     const int nE = c.count_g + c.r;
     size_t sm = (c.mode == UPD_SELECT) ? ((size_t)nE * 8 + (size_t)L.cmax * 4 + (size_t)nE + 16) : 0;
+    LaunchScope scope(st, LOLA_KERNEL_SELECT, s);
     k_select<<<U, 256, sm, s>>>(L, c);
-    st->launches++;
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   }
+  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
   k_update<T, DPL><<<U, kUpdThreads, update_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
-  st->launches++;
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
@@ -219,15 +242,24 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
   else rc = cfg->head_dim == 128 ? set_smem_attrs<float, 4>(L.D) : set_smem_attrs<float, 2>(L.D);
   if (rc == LOLA_OK && cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 9 * 16384 + 4 * 16384 + 64) != cudaSuccess)
     rc = LOLA_ERR_CUDA;
-  cudaStream_t s = (cudaStream_t)stream;
-  if (rc == LOLA_OK && cudaMemsetAsync(b, 0, lay.total, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
-  const size_t U = (size_t)cfg->batch * cfg->n_kv_heads;
-  // positions -1, scores and thresholds NaN (all-ones bit pattern)
-  if (rc == LOLA_OK && cfg->sparse > 0 && cudaMemsetAsync(L.gpos, 0xFF, U * cfg->sparse * 4, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
-  if (rc == LOLA_OK && cudaMemsetAsync(L.score, 0xFF, U * ((size_t)cfg->sparse + cfg->max_chunk) * 4, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
-  if (rc == LOLA_OK && cudaMemsetAsync(L.thr, 0xFF, U * 2 * 4, s) != cudaSuccess) rc = LOLA_ERR_CUDA;
+  if (rc == LOLA_OK) rc = lola_reset_state(st, stream);
   if (rc != LOLA_OK) { delete st; return rc; }
   *out = st;
+  return LOLA_OK;
+}
+
+int lola_reset_state(lola_state* st, void* stream) {
+  if (!st) return LOLA_ERR_ARG;
+  const lola_config& c = st->cfg;
+  const Layer& L = st->L;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t U = (size_t)c.batch * c.n_kv_heads;
+  if (cudaMemsetAsync(st->base, 0, st->lay.total, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  // positions -1, scores and thresholds NaN (all-ones bit pattern)
+  if (c.sparse > 0 && cudaMemsetAsync(L.gpos, 0xFF, U * c.sparse * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (cudaMemsetAsync(L.score, 0xFF, U * ((size_t)c.sparse + c.max_chunk) * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (cudaMemsetAsync(L.thr, 0xFF, U * 2 * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  st->n_seen = 0;
   return LOLA_OK;
 }
 
@@ -404,11 +436,41 @@ int lola_write_state(lola_state* st, const lola_state_view* v, void* stream) {
   return LOLA_OK;
 }
 
+int lola_profile_enable(lola_state* st, int enable) {
+  if (!st) return LOLA_ERR_ARG;
+  st->profiling = enable != 0;
+  return LOLA_OK;
+}
+
+int lola_profile_read(lola_state* st, double* ms_by_kind, int64_t* launches_by_kind, void* stream) {
+  if (!st || !ms_by_kind || !launches_by_kind) return LOLA_ERR_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LOLA_ERR_CUDA;
+  for (int i = 0; i < LOLA_N_KERNEL_KINDS; ++i) { ms_by_kind[i] = 0.0; launches_by_kind[i] = 0; }
+  int rc = LOLA_OK;
+  for (ProfRecord& r : st->records) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess) rc = LOLA_ERR_CUDA;
+    else if (r.kind >= 0 && r.kind < LOLA_N_KERNEL_KINDS) { ms_by_kind[r.kind] += ms; launches_by_kind[r.kind]++; }
+    st->pool.push_back(r);
+  }
+  st->records.clear();
+  return rc;
+}
+
 int64_t lola_launch_count(const lola_state* st) { return st ? st->launches : -1; }
 int64_t lola_tokens_seen(const lola_state* st) { return st ? st->n_seen : -1; }
 
+int lola_set_tokens_seen(lola_state* st, int64_t n_seen) {
+  if (!st) return LOLA_ERR_ARG;
+  if (n_seen < 0 || n_seen > 0x7fffffffLL) return LOLA_ERR_SHAPE;
+  st->n_seen = n_seen;
+  return LOLA_OK;
+}
+
 int lola_destroy_state(lola_state* st) {
   if (!st) return LOLA_ERR_ARG;
+  for (auto* v : {&st->records, &st->pool})
+    for (ProfRecord& r : *v) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   delete st;
   return LOLA_OK;
 }
