@@ -137,6 +137,34 @@ int lola_prefill_chunk(lola_state* st, const void* q, const void* k, const void*
  * Errors: ARG, ALIGN, CUDA.                                                                     */
 int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v, void* out, void* stream);
 
+/* lola_decode_step for callers that cannot provide scratch memory at call time.  The paper has no
+ * counterpart: this is a packaging variant of the generation step above, same arguments, same
+ * results.
+ *
+ * Who needs it: code that runs where device allocation is closed - a serving loop whose engine has
+ * handed all device memory to its own arena and forbids cudaMalloc after start-up, or a plug-in
+ * that only receives the persistent memories (H, s, the caches) from its host application.  The
+ * step passes small per-unit work lists from its selection kernel to its update kernel (which pairs
+ * to fold, which pair moves to which slot).  lola_decode_step keeps them in the caller's state
+ * buffer; this variant keeps them in a device array that is part of the library image, so they
+ * exist without anybody allocating them.
+ *
+ * Limits: batch * n_kv_heads <= LOLA_STATIC_MAX_UNITS and batch * n_kv_heads * max_chunk <=
+ * LOLA_STATIC_MAX_LIST_ENTRIES, otherwise LOLA_ERR_SIZE and nothing is enqueued.  The array takes
+ * (3 * LOLA_STATIC_MAX_LIST_ENTRIES + 4 * LOLA_STATIC_MAX_UNITS) * 4 bytes = 832 KiB on every GPU
+ * that loads the library, until the process exits.
+ * Set-up: the first call on each device looks up the array's device address (a host-side query,
+ * no allocation, with that device current); make that first call outside any stream capture.
+ * Sharing: all states and all calls on a device use the same array and it keeps the last call's
+ * contents.  Nothing in it has to start at zero (each step writes every entry before reading it),
+ * but two calls that overlap on the GPU (different streams, or different states on different
+ * streams) race on it: serialise them.
+ * The call itself allocates nothing: no cudaMalloc, cudaFree, or allocating library routine.
+ * Errors: as lola_decode_step, plus SIZE.                                                        */
+#define LOLA_STATIC_MAX_UNITS 4096
+#define LOLA_STATIC_MAX_LIST_ENTRIES 65536
+int lola_decode_step_static(lola_state* st, const void* q, const void* k, const void* v, void* out, void* stream);
+
 /* Same two operations for callers whose tensors live in HOST memory.  `staging_dev` is a device
  * buffer of at least lola_staging_bytes(cfg, n_tokens) bytes (256-byte aligned) that the call uses
  * for the device copies of q, k, v and out; inputs are copied in, the step runs, out is copied back

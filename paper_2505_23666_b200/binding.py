@@ -56,6 +56,7 @@ def _load() -> C.CDLL:
         "lola_init_state": (C.c_int, [cfgp, vp, vp, sz, vp, C.POINTER(vp)]),
         "lola_prefill_chunk": (C.c_int, [vp, vp, vp, vp, i32, vp, vp]),
         "lola_decode_step": (C.c_int, [vp, vp, vp, vp, vp, vp]),
+        "lola_decode_step_static": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "lola_staging_bytes": (sz, [cfgp, i32]),
         "lola_prefill_chunk_host": (C.c_int, [vp, vp, vp, vp, i32, vp, vp, sz, vp]),
         "lola_decode_step_host": (C.c_int, [vp, vp, vp, vp, vp, vp, sz, vp]),
@@ -77,7 +78,7 @@ def _load() -> C.CDLL:
 
 
 _lib = _load()
-EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_decode_step", "lola_staging_bytes",
+EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_decode_step", "lola_decode_step_static", "lola_staging_bytes",
            "lola_prefill_chunk_host", "lola_decode_step_host", "lola_read_state", "lola_write_state",
            "lola_reset_state", "lola_profile_enable", "lola_profile_read", "lola_launch_count", "lola_tokens_seen", "lola_set_tokens_seen", "lola_destroy_state", "lola_strerror"]
 
@@ -110,6 +111,12 @@ def lola_prefill_chunk(st: int, q: int, k: int, v: int, n_tokens: int, out: int,
 
 def lola_decode_step(st: int, q: int, k: int, v: int, out: int, stream: int) -> int:
     return _lib.lola_decode_step(st, q, k, v, out, stream)
+
+
+def lola_decode_step_static(st: int, q: int, k: int, v: int, out: int, stream: int) -> int:
+    """lola_decode_step with the step's work lists in the library's own static device array (for callers
+    that cannot supply scratch memory); limited to LOLA_STATIC_MAX_UNITS units."""
+    return _lib.lola_decode_step_static(st, q, k, v, out, stream)
 
 
 def lola_prefill_chunk_host(st, q_host, k_host, v_host, n_tokens, out_host, staging_dev, staging_bytes, stream) -> int:

@@ -475,6 +475,49 @@ int lola_destroy_state(lola_state* st) {
   return LOLA_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Generation step whose per-call work lists live in library-owned static device memory.
+//
+// g_static_lists is a host-side stand-in for the device array: its address means nothing to a
+// kernel.  The device address is resolved once per device with cudaGetSymbolAddress and handed
+// to the kernels through the Layer block.
+// three work lists of LOLA_STATIC_MAX_LIST_ENTRIES ints, then 4 counters per unit
+static __device__ __align__(256) int g_static_lists[3 * LOLA_STATIC_MAX_LIST_ENTRIES + 4 * LOLA_STATIC_MAX_UNITS];
+
+static int* static_lists_for_current_device(int* rc_out) {
+  static int* ptrs[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *rc_out = LOLA_ERR_CUDA; return nullptr; }
+  if (!ptrs[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_lists) != cudaSuccess || !p) { *rc_out = LOLA_ERR_CUDA; return nullptr; }
+    ptrs[dev] = (int*)p;
+  }
+  *rc_out = LOLA_OK;
+  return ptrs[dev];
+}
+
+int lola_decode_step_static(lola_state* st, const void* q, const void* k, const void* v, void* out, void* stream) {
+  if (!st) return LOLA_ERR_ARG;
+  const int64_t U = (int64_t)st->cfg.batch * st->cfg.n_kv_heads;
+  if (U > LOLA_STATIC_MAX_UNITS || U * st->cfg.max_chunk > LOLA_STATIC_MAX_LIST_ENTRIES) return LOLA_ERR_SIZE;
+  int rc = LOLA_OK;
+  int* base = static_lists_for_current_device(&rc);
+  if (!base) return rc;
+  // Same kernels, same launches as lola_decode_step; only the four work-list pointers differ.
+  // Every entry a kernel reads in a step is written earlier in the same step (the selection kernel
+  // fills the lists and both counters before the update kernel reads them), so nothing has to be
+  // cleared between calls even though the array keeps the previous call's contents.
+  const Layer saved = st->L;
+  st->L.fold_idx = base;
+  st->L.move_src = base + LOLA_STATIC_MAX_LIST_ENTRIES;
+  st->L.move_dst = base + 2 * LOLA_STATIC_MAX_LIST_ENTRIES;
+  st->L.counts = base + 3 * LOLA_STATIC_MAX_LIST_ENTRIES;
+  rc = lola_decode_step(st, q, k, v, out, stream);
+  st->L = saved;                       // kernel arguments were copied at launch
+  return rc;
+}
+
 const char* lola_strerror(int code) {
   switch (code) {
     case LOLA_OK: return "ok";
