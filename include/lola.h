@@ -54,6 +54,10 @@ typedef enum { LOLA_F32 = 0, LOLA_BF16 = 1 } lola_dtype;
  *   LOLA_PHI_EXP:     [exp(u), exp(-u)]                                              (Eq. 6).     */
 typedef enum { LOLA_PHI_SOFTMAX = 0, LOLA_PHI_EXP = 1 } lola_phi;
 
+/* config flag: run the shape-generic CUDA-core kernels even where tensor-core kernels exist (bf16,
+ * F = 64).  Both compute the same function; the flag exists for cross-checks and timing.        */
+#define LOLA_FLAG_GENERIC_KERNELS 1u
+
 typedef struct lola_config {
   int32_t batch;         /* B >= 1                                                              */
   int32_t n_q_heads;     /* Hq, multiple of n_kv_heads                                          */
@@ -69,7 +73,7 @@ typedef struct lola_config {
                             contraction and folds the rounded phi(K) (Eq. 13).                  */
   int32_t phi_kind;      /* lola_phi                                                            */
   float softmax_scale;   /* 0 => 1/sqrt(head_dim) (Eq. 2)                                       */
-  uint32_t flags;        /* reserved, must be 0                                                 */
+  uint32_t flags;        /* 0, or LOLA_FLAG_GENERIC_KERNELS                                     */
 } lola_config;
 
 /* Opaque host-side handle.  Owns no device memory. */

@@ -175,10 +175,11 @@ def lola_destroy_state(st: int) -> int:
 
 # ---- convenience holder --------------------------------------------------------------------
 def make_config(batch, n_q_heads, n_kv_heads, head_dim, feat_half, window, sparse, max_chunk,
-                dtype="bf16", phi_kind="softmax", softmax_scale=0.0) -> lola_config:
+                dtype="bf16", phi_kind="softmax", softmax_scale=0.0, generic_kernels=False) -> lola_config:
     return lola_config(batch, n_q_heads, n_kv_heads, head_dim, feat_half, window, sparse, max_chunk,
                        LOLA_BF16 if dtype == "bf16" else LOLA_F32,
-                       LOLA_PHI_EXP if phi_kind == "exp" else LOLA_PHI_SOFTMAX, float(softmax_scale), 0)
+                       LOLA_PHI_EXP if phi_kind == "exp" else LOLA_PHI_SOFTMAX, float(softmax_scale),
+                       1 if generic_kernels else 0)
 
 
 def _check(rc: int, where: str):

@@ -12,6 +12,7 @@
 #include "../../include/lola.h"
 #include "lola_generic.cuh"
 #include "lola_params.h"
+#include "lola_score_tc.cuh"
 
 using namespace lola;
 
@@ -34,7 +35,7 @@ bool config_ok(const lola_config* c) {
   if ((int64_t)c->sparse + c->max_chunk > 16384) return false;
   if (c->dtype != LOLA_F32 && c->dtype != LOLA_BF16) return false;
   if (c->phi_kind != LOLA_PHI_SOFTMAX && c->phi_kind != LOLA_PHI_EXP) return false;
-  if (!(c->softmax_scale >= 0.f) || c->flags != 0) return false;
+  if (!(c->softmax_scale >= 0.f) || (c->flags & ~(uint32_t)LOLA_FLAG_GENERIC_KERNELS) != 0) return false;
   if ((int64_t)2 * c->feat_half * c->head_dim > (int64_t)kUpdThreads * kUpdEPT) return false;
   return true;
 }
@@ -112,6 +113,7 @@ struct lola_state {
   char* base;
   int64_t n_seen;
   int64_t launches;
+  bool tensor_path = false;            // bf16, F = 64: tcgen05 kernels
   bool profiling = false;
   std::vector<ProfRecord> records;     // events in use since the last lola_profile_read
   std::vector<ProfRecord> pool;        // events ready for reuse
@@ -154,7 +156,12 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
     const int nE = c.count_g + c.r;
     dim3 grid((nE + kScoreRows - 1) / kScoreRows, U);
     LaunchScope scope(st, LOLA_KERNEL_SCORE, s);
-    k_score<T, DPL><<<grid, 256, score_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+    if (st->tensor_path) {
+      dim3 tgrid((nE + kScTile - 1) / kScTile, U);
+      k_score_tc<DPL><<<tgrid, 128, ScoreTcSmem<DPL>::bytes, s>>>(L, c);
+    } else {
+      k_score<T, DPL><<<grid, 256, score_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+    }
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   }
   if (c.mode != UPD_NONE) {
@@ -242,6 +249,13 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
   else rc = cfg->head_dim == 128 ? set_smem_attrs<float, 4>(L.D) : set_smem_attrs<float, 2>(L.D);
   if (rc == LOLA_OK && cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 9 * 16384 + 4 * 16384 + 64) != cudaSuccess)
     rc = LOLA_ERR_CUDA;
+  st->tensor_path = cfg->dtype == LOLA_BF16 && cfg->feat_half == 64 && !(cfg->flags & LOLA_FLAG_GENERIC_KERNELS);
+  if (rc == LOLA_OK && st->tensor_path) {
+    cudaError_t e = cfg->head_dim == 128
+        ? cudaFuncSetAttribute(k_score_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreTcSmem<4>::bytes)
+        : cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreTcSmem<2>::bytes);
+    if (e != cudaSuccess) rc = LOLA_ERR_CUDA;
+  }
   if (rc == LOLA_OK) rc = lola_reset_state(st, stream);
   if (rc != LOLA_OK) { delete st; return rc; }
   *out = st;

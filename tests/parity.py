@@ -43,7 +43,8 @@ def close(gpu: np.ndarray, ref: np.ndarray, tol: float, kind: str):
 
 
 class Lockstep:
-    def __init__(self, wl: Workload, rows=None, threads: int = 8, device="cuda:0", inputs: WorkloadInputs = None):
+    def __init__(self, wl: Workload, rows=None, threads: int = 8, device="cuda:0", inputs: WorkloadInputs = None,
+                 generic_kernels: bool = False):
         self.wl = wl
         self.rows = list(range(wl.batch)) if rows is None else list(rows)
         self.inputs = inputs or WorkloadInputs(wl)
@@ -52,7 +53,7 @@ class Lockstep:
         self.ocfg = config_for(wl, batch=B)
         self.oracle = LolaOracle(self.ocfg, self.inputs.W.astype(np.float64), threads=threads)
         self.cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window,
-                                       wl.sparse, max(wl.chunk, 1), dtype=wl.dtype)
+                                       wl.sparse, max(wl.chunk, 1), dtype=wl.dtype, generic_kernels=generic_kernels)
         self.layer = binding.LolaLayer(self.cfg, self.inputs.W, device=device)
         self.resyncs = 0
         self.scored_updates = 0

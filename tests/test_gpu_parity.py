@@ -53,6 +53,14 @@ def test_small_cases(name, d, F, eta, lam, C, tokens, decode, dtype):
         assert np.all(st["H"] == 0) and np.all(st["s"] == 0)
 
 
+def test_bf16_generic_kernels_flag():
+    """The CUDA-core kernels stay available in bf16 mode behind a config flag and meet the same bar."""
+    wl = small_case("bf16_generic", batch=2, n_q_heads=4, n_kv_heads=2, head_dim=128, feat_half=64, tokens=200,
+                    chunk=16, window=16, sparse=40, dtype="bf16", seed=11, decode_steps=6)
+    ls = Lockstep(wl, threads=1, generic_kernels=True)
+    drive(ls, 200, 16, 6)
+
+
 def test_exp_feature_map():
     wl = small_case("exp", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
                     dtype="f32", seed=5, decode_steps=8, scale_a=0.125)
