@@ -13,6 +13,7 @@
 #include "lola_generic.cuh"
 #include "lola_params.h"
 #include "lola_score_tc.cuh"
+#include "lola_attend_tc.cuh"
 
 using namespace lola;
 
@@ -144,7 +145,12 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   dim3 grid((L.g * c.nq + kAttRows - 1) / kAttRows, L.B * L.Hkv);
   LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
-  k_attend<T, DPL><<<grid, 256, attend_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+  if (st->tensor_path && L.g * c.nq >= 64) {
+    dim3 tgrid((L.g * c.nq + kAtM - 1) / kAtM, L.B * L.Hkv);
+    k_attend_tc<DPL><<<tgrid, 128, AttendTcSmem<DPL>::bytes, s>>>(L, c);
+  } else {
+    k_attend<T, DPL><<<grid, 256, attend_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
+  }
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
@@ -254,6 +260,10 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
     cudaError_t e = cfg->head_dim == 128
         ? cudaFuncSetAttribute(k_score_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreTcSmem<4>::bytes)
         : cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreTcSmem<2>::bytes);
+    if (e != cudaSuccess) rc = LOLA_ERR_CUDA;
+    e = cfg->head_dim == 128
+        ? cudaFuncSetAttribute(k_attend_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttendTcSmem<4>::bytes)
+        : cudaFuncSetAttribute(k_attend_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttendTcSmem<2>::bytes);
     if (e != cudaSuccess) rc = LOLA_ERR_CUDA;
   }
   if (rc == LOLA_OK) rc = lola_reset_state(st, stream);

@@ -37,6 +37,8 @@ SMALL = [
     ("bf16_d128",       128,  64,  16, 40,  16, 200,   10,   "bf16"),
     ("bf16_ragged",     128,  64,  24, 37,  20, 211,    9,   "bf16"),
     ("bf16_lam1",       128,  64,  16,  1,  16, 128,   10,   "bf16"),
+    ("bf16_tc_ragged",  128,  64,  48, 100, 64, 300,    5,   "bf16"),  # 128-row tensor-core tiles with ragged tails
+    ("bf16_tc_d64",      64,  64,  64, 200, 64, 520,    5,   "bf16"),
 ]
 
 
