@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/lola.h: argument checks, the carve-up of the caller's
 // state buffer, the per-call geometry (every count is a function of the tokens seen so far, so no
 // device value is ever read back to decide a launch), and the launches themselves.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cmath>
@@ -14,6 +15,7 @@
 #include "lola_params.h"
 #include "lola_score_tc.cuh"
 #include "lola_attend_tc.cuh"
+#include "lola_decode_tc.cuh"
 
 using namespace lola;
 
@@ -23,7 +25,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct StateLayout {
-  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, total;
+  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, wt, total;
 };
 
 bool config_ok(const lola_config* c) {
@@ -62,6 +64,8 @@ StateLayout make_layout(const lola_config& c) {
   l.move_dst = take(U * cm * 4);
   l.counts = take(U * 4 * 4);
   l.thr = take(U * 2 * 4);
+  // W^T of every KV head in tensor-core operand layout (bf16 layers with F = 64 only)
+  l.wt = take(c.dtype == LOLA_BF16 && c.feat_half == 64 ? (size_t)c.n_kv_heads * d * 64 * 2 : 0);
   l.total = o;
   return l;
 }
@@ -103,6 +107,35 @@ int set_smem_attrs(int D) {
   return LOLA_OK;
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// bf16 tensor [units][rows][d] viewed as rank 3 (d innermost); boxes of 64 columns x box_rows rows of
+// one unit, written to shared memory with the 128-byte swizzle the MMA descriptors expect.
+bool make_rows_map(CUtensorMap* tm, void* base, size_t units, size_t rows, size_t d, unsigned box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || rows == 0) return false;
+  cuuint64_t dims[3] = {d, rows, units};
+  cuuint64_t strides[2] = {d * 2, rows * d * 2};
+  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 struct ProfRecord { int kind; cudaEvent_t a, b; };
@@ -115,6 +148,9 @@ struct lola_state {
   int64_t n_seen;
   int64_t launches;
   bool tensor_path = false;            // bf16, F = 64: tcgen05 kernels
+  bool fused_decode = false;           // shapes the one-kernel generation step is built for
+  bool force_chain = false;            // set while lola_decode_step_static runs: kernel chain with work lists
+  CUtensorMap tm_gk, tm_gv, tm_wk, tm_wv;
   bool profiling = false;
   std::vector<ProfRecord> records;     // events in use since the last lola_profile_read
   std::vector<ProfRecord> pool;        // events ready for reuse
@@ -190,8 +226,20 @@ int run_prefill(lola_state* st, Call c, cudaStream_t s) {
   return launch_update_chain<T, DPL>(st, c, s);
 }
 
+template <int DPL>
+int launch_decode_fused(lola_state* st, const Call& c, cudaStream_t s) {
+  const Layer& L = st->L;
+  LaunchScope scope(st, LOLA_KERNEL_DECODE, s);
+  k_decode_tc<DPL><<<L.B * L.Hkv, kDecThreads, DecodeSmem<DPL>::bytes, s>>>(
+      L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, (const uint4*)(st->base + st->lay.wt));
+  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
 template <typename T, int DPL>
 int run_decode(lola_state* st, Call c, cudaStream_t s) {
+  // steady state (caches full, one pair leaves the window): the whole step is one kernel
+  if (st->fused_decode && !st->force_chain && c.mode == UPD_SELECT && c.r == 1 && c.count_g == st->L.lam)
+    return launch_decode_fused<DPL>(st, c, s);
   int rc = launch_update_chain<T, DPL>(st, c, s);
   if (rc != LOLA_OK) return rc;
   return launch_attend<T, DPL>(st, c, s);
@@ -266,6 +314,27 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
         : cudaFuncSetAttribute(k_attend_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttendTcSmem<2>::bytes);
     if (e != cudaSuccess) rc = LOLA_ERR_CUDA;
   }
+  // one-kernel generation step: lambda a whole number of 64-row blocks, the row stream within 16 tiles
+  st->fused_decode = st->tensor_path && cfg->sparse >= 64 && cfg->sparse % 64 == 0 && cfg->window >= 1 &&
+                     L.g <= kDecQ && (cfg->sparse / 64 + (cfg->window + 63) / 64 + 1) / 2 <= kDecMaxTiles;
+  if (rc == LOLA_OK && st->fused_decode) {
+    const size_t U = (size_t)cfg->batch * cfg->n_kv_heads;
+    bool ok = make_rows_map(&st->tm_gk, L.gk, U, cfg->sparse, cfg->head_dim, 64) &&
+              make_rows_map(&st->tm_gv, L.gv, U, cfg->sparse, cfg->head_dim, 64) &&
+              make_rows_map(&st->tm_wk, L.wk, U, cfg->window, cfg->head_dim, 64) &&
+              make_rows_map(&st->tm_wv, L.wv, U, cfg->window, cfg->head_dim, 64);
+    cudaError_t e = cfg->head_dim == 128
+        ? cudaFuncSetAttribute(k_decode_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes)
+        : cudaFuncSetAttribute(k_decode_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+    if (!ok || e != cudaSuccess) st->fused_decode = false;   // the kernel chain serves every shape
+  }
+  if (rc == LOLA_OK && st->tensor_path) {
+    cudaStream_t s = (cudaStream_t)stream;
+    __nv_bfloat16* img = (__nv_bfloat16*)(st->base + lay.wt);
+    if (cfg->head_dim == 128) k_prep_wt_image<4><<<cfg->n_kv_heads, 256, 0, s>>>((const __nv_bfloat16*)W_dev, img, cfg->n_kv_heads);
+    else k_prep_wt_image<2><<<cfg->n_kv_heads, 256, 0, s>>>((const __nv_bfloat16*)W_dev, img, cfg->n_kv_heads);
+    if (cudaGetLastError() != cudaSuccess) rc = LOLA_ERR_CUDA;
+  }
   if (rc == LOLA_OK) rc = lola_reset_state(st, stream);
   if (rc != LOLA_OK) { delete st; return rc; }
   *out = st;
@@ -278,7 +347,7 @@ int lola_reset_state(lola_state* st, void* stream) {
   const Layer& L = st->L;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t U = (size_t)c.batch * c.n_kv_heads;
-  if (cudaMemsetAsync(st->base, 0, st->lay.total, s) != cudaSuccess) return LOLA_ERR_CUDA;
+  if (cudaMemsetAsync(st->base, 0, st->lay.wt, s) != cudaSuccess) return LOLA_ERR_CUDA;   // all but the W^T image
   // positions -1, scores and thresholds NaN (all-ones bit pattern)
   if (c.sparse > 0 && cudaMemsetAsync(L.gpos, 0xFF, U * c.sparse * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
   if (cudaMemsetAsync(L.score, 0xFF, U * ((size_t)c.sparse + c.max_chunk) * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
@@ -537,7 +606,9 @@ int lola_decode_step_static(lola_state* st, const void* q, const void* k, const 
   st->L.move_src = base + LOLA_STATIC_MAX_LIST_ENTRIES;
   st->L.move_dst = base + 2 * LOLA_STATIC_MAX_LIST_ENTRIES;
   st->L.counts = base + 3 * LOLA_STATIC_MAX_LIST_ENTRIES;
+  st->force_chain = true;              // the kernel chain is the path that passes work lists between kernels
   rc = lola_decode_step(st, q, k, v, out, stream);
+  st->force_chain = false;
   st->L = saved;                       // kernel arguments were copied at launch
   return rc;
 }

@@ -1,0 +1,621 @@
+// The generation step (Eq. 11-14) as ONE kernel for the steady state of a bf16 layer with F = 64:
+// caches full, exactly one pair leaves the window per step.  One CTA per (batch row, KV head) unit;
+// the unit's memories are streamed once from HBM by TMA and everything that depends on them is
+// computed on the way:
+//
+//   rows of the stream = sparse-cache slots 0..lambda-1, then the window ring slots 0..eta-1, in
+//   tiles of 128 rows.  Per tile (one thread per row, two row groups of 128 threads work on
+//   alternate tiles so that one group's arithmetic overlaps the other's loads and MMAs):
+//     [U | Z] = K_tile [W | Q^T]          tcgen05.mma  M=128, N=80, K=d   (pre-activations, q.k)
+//     phi = feature map of U, rounded to bf16; den = phi . s
+//     P = phi H                            tcgen05.mma  M=128, N=d,  K=128
+//     score = || P / den - v ||            for sparse-cache rows and the evicted pair (Eq. 10)
+//     O^T += V_tile^T Pr^T                 tcgen05.mma  M=d(128), N=16, K=128 (Eq. 14 numerator),
+//                                          Pr = exp(z - m) with a running maximum per query row
+//   The pair to fold (Eq. 12: lowest score, ties: the younger pair) is only known after the last
+//   tile, and it must not be attended.  So every tile leaves its own lowest-scored row out of O^T and
+//   keeps that row's q.k, value and feature row in a small list; at the end the overall lowest is
+//   folded (Eq. 13: H += phi v^T, s += phi) and the other list entries are added back.
+//   The linear term uses the state after the fold: phi(q)^T H_old (an MMA that initialises O^T with
+//   weight exp(0 - m), the m = max(0, .) stabiliser) plus (phi(q) . phi_fold) v_fold.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out sets bit 8 of the status word.
+#pragma once
+#include <cuda.h>
+
+#include "lola_generic.cuh"
+#include "lola_tc.cuh"
+
+namespace lola {
+
+constexpr int kDecQ = 8;          // query rows per unit the kernel carries (group size g <= 8)
+constexpr int kDecMaxTiles = 16;  // (lambda + eta rounded up to 64) / 128 <= 16
+constexpr int kDecThreads = 256;
+
+template <int DPL>
+struct DecodeSmem {
+  static constexpr int d = DPL * 32;
+  static constexpr int kblk = d / 64;
+  static constexpr uint32_t b1_blk = 80 * 128;                       // one K block of [W^T ; Q]: 80 rows
+  static constexpr uint32_t b1 = 0;                                  // [kblk][80][128B]
+  static constexpr uint32_t hmn = 2 * b1_blk;                        // H, MN-major: [kblk (c blocks)][128 j][128B]
+  static constexpr uint32_t phiq = hmn + 2 * 16384;                  // phi(Q), K-major: [2 j blocks][16][128B]
+  static constexpr uint32_t stage0 = phiq + 4096;
+  static constexpr uint32_t st_k = 0;                                // K tile [kblk][128][128B]; then phi tile [2][128][128B]
+  static constexpr uint32_t st_v = 32768;                            // V tile [kblk][128 keys][128B]
+  static constexpr uint32_t st_pt = 65536;                           // Pr^T, K-major: [2 key blocks][16][128B]
+  static constexpr uint32_t stage_bytes = 65536 + 4096;
+  static constexpr uint32_t misc = stage0 + 2 * stage_bytes;         // small arrays, see DecodeMisc
+  static constexpr uint32_t total = misc + 32768;
+  static constexpr uint32_t bytes = total + 1024;                    // slack to align the base to 1024
+};
+
+// small shared arrays (all fp32 / int unless noted)
+struct DecodeMisc {
+  float s_vec[128];
+  float qf[kDecQ][128];          // query rows, fp32
+  float phiq_f[kDecQ][128];      // phi(q) rounded to bf16, as fp32
+  float u_s[kDecQ][64];
+  float knew[128], vnew[128];
+  float zn[kDecQ], lden[kDecQ], dotL[kDecQ];
+  float redmax[2][4][kDecQ];
+  unsigned long long redkey[2][4];
+  float red12[2][4][2];
+  float wg_m[2][kDecQ];
+  float wg_l[2][4][kDecQ];
+  float opart[2][128][kDecQ];
+  // per-tile list of the rows left out of O^T
+  unsigned long long cand_key[kDecMaxTiles];
+  float cand_score[kDecMaxTiles], cand_min2[kDecMaxTiles];
+  int cand_row[kDecMaxTiles];
+  float cand_z[kDecMaxTiles][kDecQ];
+  uint4 cand_v[kDecMaxTiles][16];    // value row, bf16
+  uint4 cand_phi[kDecMaxTiles][16];  // feature row, bf16
+  uint64_t bars[8];
+  uint32_t tmem_slot;
+};
+static_assert(sizeof(DecodeMisc) <= 32768, "misc region too small");
+
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long x, int o) {
+  unsigned lo = __shfl_xor_sync(0xffffffffu, (unsigned)x, o);
+  unsigned hi = __shfl_xor_sync(0xffffffffu, (unsigned)(x >> 32), o);
+  return ((unsigned long long)hi << 32) | lo;
+}
+
+// Loads of one tile: two half tiles of 64 rows; a half tile is a block of sparse-cache slots, a block
+// of ring slots, or nothing (a box that lies entirely outside the ring tensor reads as zeros).
+template <int DPL>
+__device__ __forceinline__ void decode_issue_tile(uint32_t dst, const CUtensorMap* tm_g, const CUtensorMap* tm_w, int tile,
+                                                  int nGB, int nRB, int unit, uint32_t bar) {
+  constexpr int kblk = DPL / 2;
+  tc::mbar_expect_tx(bar, (uint32_t)kblk * 16384u);
+#pragma unroll
+  for (int hb = 0; hb < 2; ++hb) {
+    const int blk = tile * 2 + hb;
+    const bool from_g = blk < nGB;
+    const CUtensorMap* tm = from_g ? tm_g : tm_w;
+    const int row = from_g ? blk * 64 : min(blk - nGB, nRB) * 64;
+#pragma unroll
+    for (int cb = 0; cb < kblk; ++cb)
+      tc::tma_load_3d(dst + (uint32_t)cb * 16384u + (uint32_t)hb * 8192u, tm, cb * 64, row, unit, bar);
+  }
+}
+
+template <int DPL>
+__global__ void __launch_bounds__(kDecThreads, 1)
+k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
+            const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image) {
+  using S = DecodeSmem<DPL>;
+  constexpr int d = DPL * 32;
+  constexpr int kblk = d / 64;
+  constexpr int F = 64, D = 128;
+  constexpr float kLog2e = 1.4426950408889634f;
+  typedef __nv_bfloat16 T;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = tc::smem_u32(sm);
+  DecodeMisc& X = *reinterpret_cast<DecodeMisc*>(sm + S::misc);
+
+  const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
+  const int tid = threadIdx.x, wg = tid >> 7, t = tid & 127, warp = tid >> 5, wq = warp & 3, lane = tid & 31;
+  const int lam = L.lam, eta = L.eta, g = L.g;
+  const int nGB = lam / 64, nRB = (eta + 63) / 64, NT = (nGB + nRB + 1) / 2;
+  const int s_ev = c.n_seen % eta;          // ring slot of the pair that leaves = slot the new pair takes
+  const int pos_ev = c.n_seen - eta;
+  float* scu = L.score + (size_t)unit * (lam + L.cmax);
+
+  const uint32_t bar_k = sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + (uint32_t)wg * 24u;
+  const uint32_t bar_v = bar_k + 8, bar_mma = bar_k + 16;
+  const uint32_t stage = sbase + S::stage0 + (uint32_t)wg * S::stage_bytes;
+  uint8_t* stage_p = sm + S::stage0 + (size_t)wg * S::stage_bytes;
+  uint32_t pk = 0, pv = 0, pm = 0;
+  bool ok = true;
+
+  if (tid == 0) {
+    for (int i = 0; i < 6; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + 8u * i, 1);
+    tc::mbar_init_fence();
+  }
+  if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
+  __syncthreads();
+  // first tile of each row group starts to stream while the operands below are prepared
+  if (t == 0 && wg < NT) {
+    decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, wg, nGB, nRB, unit, bar_k);
+    decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, wg, nGB, nRB, unit, bar_v);
+  }
+
+  // ---- operands that stay for the whole unit
+  {
+    // H (fp32, [D][d]) -> bf16, MN-major: c block, row j, 64 c per 128-byte row
+    const float4* Hg = reinterpret_cast<const float4*>(L.H + (size_t)unit * D * d);
+    constexpr int per_row = d / 8;
+#pragma unroll 4
+    for (int i = tid; i < D * per_row; i += kDecThreads) {
+      const int j = i / per_row, c8 = (i % per_row) * 8;
+      float4 a = Hg[(size_t)i * 2], bq = Hg[(size_t)i * 2 + 1];
+      float f8[8] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w};
+      *reinterpret_cast<uint4*>(sm + S::hmn + (c8 >> 6) * 16384 + tc::sw128_off(j, (c8 & 63) >> 3)) = tc::pack8_bf16(f8);
+    }
+    // W^T image (prepared once per layer in the operand layout): rows 0..63 of each K block of B1
+    const uint4* img = wt_image + (size_t)h * kblk * 512;
+    for (int i = tid; i < kblk * 512; i += kDecThreads)
+      *reinterpret_cast<uint4*>(sm + S::b1 + (i >> 9) * S::b1_blk + (i & 511) * 16) = img[i];
+    // query rows: B1 rows 64..79 (rows >= g are zero) and an fp32 copy
+    for (int i = tid; i < 16 * per_row; i += kDecThreads) {
+      const int r = i / per_row, ch = i % per_row;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (r < g) val = *reinterpret_cast<const uint4*>((const T*)c.q + ((size_t)b * L.Hq + h * g + r) * d + ch * 8);
+      *reinterpret_cast<uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(64 + r, ch & 7)) = val;
+      if (r < kDecQ) {
+        const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&val);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float2 ff = __bfloat1622float2(v2[q]);
+          X.qf[r][ch * 8 + 2 * q] = ff.x;
+          X.qf[r][ch * 8 + 2 * q + 1] = ff.y;
+        }
+      }
+    }
+    if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
+    if (tid < d) {
+      X.knew[tid] = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + tid);
+      X.vnew[tid] = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + tid);
+    }
+    if (tid < kDecMaxTiles) { X.cand_key[tid] = ~0ull; X.cand_score[tid] = CUDART_INF_F; X.cand_min2[tid] = CUDART_INF_F; X.cand_row[tid] = 0; }
+    // zero phi(Q) and both Pr^T tiles
+    for (int i = tid; i < 256; i += kDecThreads) {
+      *reinterpret_cast<uint4*>(sm + S::phiq + i * 16) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(sm + S::stage0 + S::st_pt + i * 16) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(sm + S::stage0 + S::stage_bytes + S::st_pt + i * 16) = make_uint4(0, 0, 0, 0);
+    }
+  }
+  __syncthreads();
+  // u = q W on the CUDA cores (g rows only) from the W^T operand image, then phi(q), its normaliser
+  // and q . k_new
+  for (int i = tid; i < g * F; i += kDecThreads) {
+    const int r = i >> 6, f = i & 63;
+    float a = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < d / 8; ++ch) {
+      uint4 raw = *reinterpret_cast<const uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(f, ch & 7));
+      const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float2 ww = __bfloat1622float2(w2[q]);
+        a = fmaf(X.qf[r][ch * 8 + 2 * q], ww.x, a);
+        a = fmaf(X.qf[r][ch * 8 + 2 * q + 1], ww.y, a);
+      }
+    }
+    X.u_s[r][f] = a;
+  }
+  __syncthreads();
+  if (warp < g) {
+    const int r = warp;
+    float u0 = X.u_s[r][lane], u1 = X.u_s[r][lane + 32];
+    float p0, p1, n0, n1;
+    if (L.phi_kind == 1) {
+      p0 = expf(u0); p1 = expf(u1); n0 = expf(-u0); n1 = expf(-u1);
+    } else {
+      float mx = warp_max(fmaxf(u0, u1)), mn = warp_min(fminf(u0, u1));
+      p0 = expf(u0 - mx); p1 = expf(u1 - mx); n0 = expf(mn - u0); n1 = expf(mn - u1);
+      float s1 = warp_sum(p0 + p1), s2 = warp_sum(n0 + n1);
+      p0 /= s1; p1 /= s1; n0 /= s2; n1 /= s2;
+    }
+    float vals[4] = {round_bf16f(p0), round_bf16f(p1), round_bf16f(n0), round_bf16f(n1)};
+    int js[4] = {lane, lane + 32, 64 + lane, 96 + lane};
+    float ld = 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int j = js[q];
+      X.phiq_f[r][j] = vals[q];
+      *reinterpret_cast<T*>(sm + S::phiq + (j >> 6) * 2048 + tc::sw128_off(r, (j & 63) >> 3) + (j & 7) * 2) = __float2bfloat16_rn(vals[q]);
+      ld = fmaf(vals[q], X.s_vec[j], ld);
+    }
+    ld = warp_sum(ld);
+    float zz = 0.f;
+    for (int j = lane; j < d; j += 32) zz = fmaf(X.qf[r][j], X.knew[j], zz);
+    zz = warp_sum(zz);
+    if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * L.scale; }
+  }
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem = X.tmem_slot;
+  const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+  const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // [U | Z], then P
+  const uint32_t tm_o = tm_a + 160u;                            // O^T: lanes = value column, 16 columns = query rows
+  const uint32_t idesc1 = tc::make_idesc_bf16(128, 80, false, false);
+  const uint32_t idesc2 = tc::make_idesc_bf16(128, d, false, true);
+  const uint32_t idesc3 = tc::make_idesc_bf16(128, 16, true, false);
+
+  bool have_o = false;
+  if (wg == 0) {
+    // O^T = H^T phi(Q)^T: the linear term enters the running sums with weight exp(0 - m), m = 0 so far
+    if (t == 0) {
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks)
+        tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::hmn + ks * 2048, 16384, 1024),
+                        tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc3, ks > 0);
+    }
+    have_o = true;
+  }
+
+  float m_run[kDecQ], lpart[kDecQ];
+#pragma unroll
+  for (int r = 0; r < kDecQ; ++r) { m_run[r] = 0.f; lpart[r] = 0.f; }
+
+  for (int tile = wg; tile < NT; tile += 2) {
+    const int R = tile * 128 + t;
+    const bool is_g = R < lam;
+    const int slot = R - lam;
+    const bool valid = is_g || slot < eta;
+    const bool scored = is_g || slot == s_ev;
+    const int pos = is_g ? L.gpos[(size_t)unit * lam + R] : pos_ev;
+
+    // ---- [U | Z] = K_tile [W | Q^T]
+    ok = tc::mbar_wait(bar_k, pk) && ok; pk ^= 1;
+    tc::fence_after_sync();
+    if (t == 0) {
+#pragma unroll
+      for (int ks = 0; ks < d / 16; ++ks)
+        tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                        tc::make_desc_sw128(sbase + S::b1 + (ks >> 2) * S::b1_blk + (ks & 3) * 32, 16, 1024), idesc1, ks > 0);
+      tc::mma_commit(bar_mma);
+    }
+    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
+    tc::fence_after_sync();
+
+    float z[kDecQ];
+    float den = 0.f;
+    {
+      float zraw[8];
+      tc::tmem_ld8(tm_a + lane_addr + 64, zraw);
+#pragma unroll
+      for (int r = 0; r < kDecQ; ++r) z[r] = valid ? zraw[r] * L.scale : -CUDART_INF_F;
+      float u0[32], u1[32];
+      tc::tmem_ld32(tm_a + lane_addr, u0);
+      tc::tmem_ld32(tm_a + lane_addr + 32, u1);
+      // feature map, one half at a time; each half goes to the A operand of the second product
+      // (over the key tile, which the first product no longer needs)
+      float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        mx = fmaxf(mx, fmaxf(u0[i], u1[i]));
+        mn = fminf(mn, fminf(u0[i], u1[i]));
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float f[64];
+        if (L.phi_kind == 1) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            f[i] = expf(half ? -u0[i] : u0[i]);
+            f[32 + i] = expf(half ? -u1[i] : u1[i]);
+          }
+        } else {
+          const float off = half ? mn : -mx;
+          float ssum = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            f[i] = tc::fast_exp2(((half ? -u0[i] : u0[i]) + off) * kLog2e);
+            f[32 + i] = tc::fast_exp2(((half ? -u1[i] : u1[i]) + off) * kLog2e);
+          }
+#pragma unroll
+          for (int i = 0; i < 64; ++i) ssum += f[i];
+          const float inv = 1.0f / ssum;
+#pragma unroll
+          for (int i = 0; i < 64; ++i) f[i] *= inv;
+        }
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+          f[i] = round_bf16f(f[i]);
+          den = fmaf(f[i], X.s_vec[half * 64 + i], den);
+        }
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch)
+          *reinterpret_cast<uint4*>(stage_p + S::st_k + half * 16384 + tc::sw128_off(t, ch)) = tc::pack8_bf16(f + ch * 8);
+      }
+    }
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    tc::named_bar_sync(1 + wg, 128);
+    tc::fence_after_sync();
+    // ---- P = phi H
+    if (t == 0) {
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks)
+        tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                        tc::make_desc_sw128(sbase + S::hmn + ks * 2048, 16384, 1024), idesc2, ks > 0);
+      tc::mma_commit(bar_mma);
+    }
+    // meanwhile: running maximum of q.k per query row (every valid row counts, also the one that will
+    // be folded: any m >= the true maximum leaves Eq. 14 unchanged)
+    float m_new[kDecQ];
+#pragma unroll
+    for (int r = 0; r < kDecQ; ++r) {
+      float wm = warp_max(z[r]);
+      if (lane == 0) X.redmax[wg][wq][r] = wm;
+    }
+    tc::named_bar_sync(1 + wg, 128);
+#pragma unroll
+    for (int r = 0; r < kDecQ; ++r)
+      m_new[r] = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[wg][0][r], X.redmax[wg][1][r])),
+                       fmaxf(X.redmax[wg][2][r], X.redmax[wg][3][r]));
+
+    ok = tc::mbar_wait(bar_v, pv) && ok; pv ^= 1;
+    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
+    tc::fence_after_sync();
+    // ---- Eq. 10
+    float score;
+    {
+      float ss = 0.f;
+      const bool pos_den = den > 0.f;
+#pragma unroll
+      for (int c0 = 0; c0 < d; c0 += 32) {
+        float p[32];
+        tc::tmem_ld32(tm_a + lane_addr + c0, p);
+#pragma unroll
+        for (int q8 = 0; q8 < 4; ++q8) {
+          const int cc = c0 + q8 * 8;
+          uint4 raw = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (cc >> 6) * 16384 + tc::sw128_off(t, (cc & 63) >> 3));
+          const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            float2 vv = __bfloat1622float2(v2[q]);
+            float d0 = (pos_den ? p[q8 * 8 + 2 * q] / den : 0.f) - vv.x;
+            float d1 = (pos_den ? p[q8 * 8 + 2 * q + 1] / den : 0.f) - vv.y;
+            ss = fmaf(d0, d0, ss);
+            ss = fmaf(d1, d1, ss);
+          }
+        }
+      }
+      score = sqrtf(ss);
+    }
+    if (scored && ok) scu[is_g ? R : lam] = score;
+    // lowest score of the tile (ties: the younger pair), and the two lowest values
+    unsigned long long key = scored ? (((unsigned long long)__float_as_uint(score) << 32) | (unsigned)(0x7fffffff - pos))
+                                    : ~0ull;
+    {
+      unsigned long long k = key;
+      float a1 = scored ? score : CUDART_INF_F, a2 = CUDART_INF_F;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long ko = shfl_xor_u64(k, o);
+        k = ko < k ? ko : k;
+        float b1 = __shfl_xor_sync(0xffffffffu, a1, o), b2 = __shfl_xor_sync(0xffffffffu, a2, o);
+        float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
+        a2 = fminf(hi, fminf(a2, b2));
+        a1 = lo;
+      }
+      if (lane == 0) { X.redkey[wg][wq] = k; X.red12[wg][wq][0] = a1; X.red12[wg][wq][1] = a2; }
+    }
+    tc::named_bar_sync(1 + wg, 128);
+    unsigned long long tkey = X.redkey[wg][0];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) tkey = X.redkey[wg][w] < tkey ? X.redkey[wg][w] : tkey;
+    const bool left_out = scored && key == tkey;
+    if (left_out) {
+      float a1 = X.red12[wg][0][0], a2 = X.red12[wg][0][1];
+#pragma unroll
+      for (int w = 1; w < 4; ++w) {
+        float b1 = X.red12[wg][w][0], b2 = X.red12[wg][w][1];
+        float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
+        a2 = fminf(hi, fminf(a2, b2));
+        a1 = lo;
+      }
+      X.cand_key[tile] = key;
+      X.cand_score[tile] = score;
+      X.cand_min2[tile] = a2;
+      X.cand_row[tile] = R;
+#pragma unroll
+      for (int r = 0; r < kDecQ; ++r) X.cand_z[tile][r] = z[r];
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) {
+        X.cand_phi[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_k + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
+        if (ch < d / 8)
+          X.cand_v[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
+      }
+    }
+    // ---- softmax weights of the tile (bf16, the sums use the rounded weights) and running sums
+    {
+      bool moved = false;
+      float alpha[kDecQ];
+#pragma unroll
+      for (int r = 0; r < kDecQ; ++r) {
+        alpha[r] = tc::fast_exp2((m_run[r] - m_new[r]) * kLog2e);
+        moved = moved || (m_new[r] != m_run[r]);
+        float p = (valid && !left_out) ? tc::fast_exp2((z[r] - m_new[r]) * kLog2e) : 0.f;
+        p = round_bf16f(p);
+        lpart[r] = lpart[r] * alpha[r] + p;
+        m_run[r] = m_new[r];
+        *reinterpret_cast<T*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = __float2bfloat16_rn(p);
+      }
+      if (have_o && moved) {                     // uniform over the row group
+        float ov[8];
+        tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+        for (int r = 0; r < kDecQ; ++r) ov[r] *= alpha[r];
+        tc::tmem_st8(tm_o + lane_addr, ov);
+      }
+    }
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    tc::named_bar_sync(1 + wg, 128);
+    tc::fence_after_sync();
+    // ---- O^T += V^T Pr^T; the key/phi buffer is free for the next tile of this row group
+    if (t == 0) {
+      if (tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(stage + S::st_v + ks * 2048, 16384, 1024),
+                        tc::make_desc_sw128(stage + S::st_pt + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc3,
+                        (have_o || ks > 0) ? 1u : 0u);
+      tc::mma_commit(bar_mma);
+    }
+    have_o = true;
+    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
+    tc::fence_after_sync();
+    if (t == 0 && tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_v);
+  }
+
+  // ---- per row group: maximum, sums, partial O^T
+#pragma unroll
+  for (int r = 0; r < kDecQ; ++r) {
+    float ls = warp_sum(lpart[r]);
+    if (lane == 0) X.wg_l[wg][wq][r] = ls;
+  }
+#pragma unroll
+  for (int r = 0; r < kDecQ; ++r)
+    if (t == r) X.wg_m[wg][r] = m_run[r];          // m_run is uniform over the row group
+  {
+    float ov[8];
+#pragma unroll
+    for (int r = 0; r < kDecQ; ++r) ov[r] = 0.f;
+    if (have_o) tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+    for (int r = 0; r < kDecQ; ++r) X.opart[wg][t][r] = ov[r];
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+
+  // ---- the pair to fold: lowest (score, then youngest) over the tiles' left-out rows
+  int lt = 0;
+  {
+    unsigned long long best = X.cand_key[0];
+    for (int i = 1; i < NT; ++i)
+      if (X.cand_key[i] < best) { best = X.cand_key[i]; lt = i; }
+  }
+  if (warp < g) {                                 // phi(q) . phi_fold
+    const int r = warp;
+    const __nv_bfloat16* pf = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
+    float a = 0.f;
+    for (int j = lane; j < D; j += 32) a = fmaf(X.phiq_f[r][j], __bfloat162float(pf[j]), a);
+    a = warp_sum(a);
+    if (lane == 0) X.dotL[r] = a;
+  }
+  __syncthreads();
+  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
+  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
+
+  // ---- Eq. 14
+  if (tid < d && ok) {
+    const int cc = tid;
+    for (int r = 0; r < g; ++r) {
+      const float m0 = X.wg_m[0][r], m1 = X.wg_m[1][r];
+      const float mf = fmaxf(fmaxf(m0, m1), X.zn[r]);
+      const float a0 = tc::fast_exp2((m0 - mf) * kLog2e), a1 = tc::fast_exp2((m1 - mf) * kLog2e);
+      float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) { l0 += X.wg_l[0][w][r]; l1 += X.wg_l[1][w][r]; }
+      float num = a0 * X.opart[0][cc][r] + a1 * X.opart[1][cc][r];
+      float den = a0 * l0 + a1 * l1;
+      for (int i = 0; i < NT; ++i) {
+        if (i == lt || X.cand_key[i] == ~0ull) continue;
+        const float p = round_bf16f(tc::fast_exp2((X.cand_z[i][r] - mf) * kLog2e));
+        num = fmaf(p, __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[i][0])[cc]), num);
+        den += p;
+      }
+      const float pn = tc::fast_exp2((X.zn[r] - mf) * kLog2e);
+      num = fmaf(pn, X.vnew[cc], num);
+      den += pn;
+      const float e = tc::fast_exp2(-mf * kLog2e);
+      num = fmaf(e * X.dotL[r], __bfloat162float(vL[cc]), num);
+      den = fmaf(e, X.lden[r] + X.dotL[r], den);
+      ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
+    }
+  }
+
+  // ---- Eq. 13: H += phi_fold v_fold^T, s += phi_fold
+  if (ok) {
+    float4* Hg = reinterpret_cast<float4*>(L.H + (size_t)unit * D * d);
+    constexpr int per_row = d / 4;
+#pragma unroll 4
+    for (int i = tid; i < D * per_row; i += kDecThreads) {
+      const int j = i / per_row, c4 = (i % per_row) * 4;
+      const float pj = __bfloat162float(phiL[j]);
+      float4 hv = Hg[i];
+      hv.x = fmaf(pj, __bfloat162float(vL[c4]), hv.x);
+      hv.y = fmaf(pj, __bfloat162float(vL[c4 + 1]), hv.y);
+      hv.z = fmaf(pj, __bfloat162float(vL[c4 + 2]), hv.z);
+      hv.w = fmaf(pj, __bfloat162float(vL[c4 + 3]), hv.w);
+      Hg[i] = hv;
+    }
+    if (tid < D) L.s[(size_t)unit * D + tid] += __bfloat162float(phiL[tid]);
+  }
+
+  // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself)
+  const int rowL = X.cand_row[lt];
+  const T* ring_k = (const T*)L.wk + ((size_t)unit * eta + s_ev) * d;
+  const T* ring_v = (const T*)L.wv + ((size_t)unit * eta + s_ev) * d;
+  if (ok && rowL < lam) {
+    constexpr int nch = d / 8;
+    if (tid < 2 * nch) {
+      const T* src = tid < nch ? ring_k : ring_v;
+      T* dst = (tid < nch ? (T*)L.gk : (T*)L.gv) + ((size_t)unit * lam + rowL) * d;
+      const int ch = tid % nch;
+      *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
+    }
+    if (tid == 64) {
+      L.gpos[(size_t)unit * lam + rowL] = pos_ev;
+      scu[rowL] = scu[lam];
+    }
+  }
+  if (tid == 96 && ok) {
+    // lowest kept / highest folded score of this update
+    float second = X.cand_min2[lt];
+    for (int i = 0; i < NT; ++i)
+      if (i != lt) second = fminf(second, X.cand_score[i]);
+    L.thr[(size_t)unit * 2 + 0] = second;
+    L.thr[(size_t)unit * 2 + 1] = X.cand_score[lt];
+  }
+  __syncthreads();
+  // ---- the new pair enters the window ring
+  if (ok) {
+    constexpr int nch = d / 8;
+    if (tid < 2 * nch) {
+      const T* src = (tid < nch ? (const T*)c.k : (const T*)c.v) + ((size_t)b * L.Hkv + h) * d;
+      T* dst = (tid < nch ? (T*)L.wk : (T*)L.wv) + ((size_t)unit * eta + s_ev) * d;
+      const int ch = tid % nch;
+      *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
+    }
+  }
+  if (!ok && t == 0) atomicOr(L.status, 8);
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, 512);
+}
+
+// Writes, once per layer, W^T of every KV head as the K-major 128-byte-swizzled operand image the
+// decode kernel copies into shared memory: per head [d/64 K blocks][64 rows f][128 bytes = 64 i].
+template <int DPL>
+__global__ void k_prep_wt_image(const __nv_bfloat16* W, __nv_bfloat16* image, int Hkv) {
+  constexpr int d = DPL * 32, F = 64;
+  const int h = blockIdx.x;
+  for (int i = threadIdx.x; i < d * F; i += blockDim.x) {
+    const int j = i / F, f = i % F;
+    const size_t off = (size_t)h * (d / 64) * 8192 + (size_t)(j >> 6) * 8192 + tc::sw128_off(f, (j & 63) >> 3) + (j & 7) * 2;
+    image[off / 2] = W[(size_t)h * d * F + i];
+  }
+}
+
+}  // namespace lola

@@ -76,12 +76,17 @@ class Lockstep:
     def decode(self, step: int, check_state: bool = True):
         q, k, v = self.inputs.decode_token(step, batch_rows=self.rows)
         L = self.layer
-        out = L.decode_step(L.to_device(q), L.to_device(k), L.to_device(v))
+        out = L.decode_step(L.to_device(q), L.to_device(k), L.to_device(v)).float().cpu().numpy()
         ref = self.oracle.decode_step(q, k, v)
-        self._cmp_out(out.float().cpu().numpy(), ref, f"decode step={step}")
         self.calls += 1
-        if check_state:
-            self.check_state(f"decode step={step}")
+        # A generation step selects first and attends afterwards, so where the two sides resolved a
+        # near-tie differently (verified against the oracle's own scores in check_state) their outputs
+        # of this step answer different, equally valid, cache contents: those units are not compared.
+        diverged = self.check_state(f"decode step={step}") if check_state else []
+        g = self.wl.group
+        for (b, h) in diverged:
+            out[b, h * g:(h + 1) * g] = ref[b, h * g:(h + 1) * g]
+        self._cmp_out(out, ref, f"decode step={step}")
 
     # ------------------------------------------------------------------ comparisons
     def _cmp_out(self, gpu, ref, where):
@@ -98,6 +103,7 @@ class Lockstep:
         assert np.array_equal(g["window_count"], o["window_count"]), f"{where}: window counts differ"
         B, Hk = g["sparse_count"].shape
         need_resync = False
+        diverged = []
         for b in range(B):
             for h in range(Hk):
                 u = self.oracle.units[b][h]
@@ -136,10 +142,12 @@ class Lockstep:
                 else:
                     self._assert_near_tie(u, set(gpos.tolist()), where, (b, h))
                     need_resync = True
+                    diverged.append((b, h))
         self.scored_updates = sum(u.n_scored_updates for row in self.oracle.units for u in row)
         if need_resync:
             self.resyncs += 1
             self.layer.write_state(o)
+        return diverged
 
     def _assert_near_tie(self, u, gpu_members: set, where, unit):
         """Membership differs: every pair on the wrong side must be a near-tie in the ORACLE's scores of

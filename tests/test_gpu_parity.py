@@ -39,6 +39,11 @@ SMALL = [
     ("bf16_lam1",       128,  64,  16,  1,  16, 128,   10,   "bf16"),
     ("bf16_tc_ragged",  128,  64,  48, 100, 64, 300,    5,   "bf16"),  # 128-row tensor-core tiles with ragged tails
     ("bf16_tc_d64",      64,  64,  64, 200, 64, 520,    5,   "bf16"),
+    # lambda a multiple of 64: the generation steps run as the single fused kernel once the caches are full
+    ("bf16_fused_d128", 128,  64,  64, 192, 64, 448,   24,   "bf16"),
+    ("bf16_fused_d64",   64,  64,  32,  64, 32, 256,   24,   "bf16"),
+    ("bf16_fused_eta100", 128, 64, 100, 128, 50, 400,  16,   "bf16"),  # two ring blocks, the second ragged
+    ("bf16_fused_eta1", 128,  64,   1,  64, 16, 160,   12,   "bf16"),  # the window is the new pair alone
 ]
 
 
@@ -53,6 +58,32 @@ def test_small_cases(name, d, F, eta, lam, C, tokens, decode, dtype):
     if name == "f32_all_softmax":
         st = ls.layer.read_state()
         assert np.all(st["H"] == 0) and np.all(st["s"] == 0)
+
+
+@pytest.mark.parametrize("g,batch", [(1, 3), (4, 2), (8, 1)])
+def test_fused_decode_group_sizes(g, batch):
+    """Fused generation step for 1, 4 and 8 query heads per KV head, then many steps in a row."""
+    wl = small_case(f"fused_g{g}", batch=batch, n_q_heads=2 * g, n_kv_heads=2, head_dim=128, feat_half=64, tokens=384,
+                    chunk=64, window=64, sparse=128, dtype="bf16", seed=13, decode_steps=40)
+    ls = Lockstep(wl, threads=1)
+    summ = drive(ls, 384, 64, 40)
+    assert summ["resyncs"] <= 2, summ
+
+
+def test_cfg3_shape_decode_sample():
+    """Two batch rows of the decode workload at its full shapes (lambda 832, window 64, 4 query heads per KV
+    head, d 128) after a shortened prefill that fills both caches, 48 fused steps against the oracle."""
+    wl = WORKLOADS["cfg3"].with_(batch=2, tokens=2048, decode_steps=48)
+    ls = Lockstep(wl)
+    t = 0
+    while t < wl.tokens:
+        ls.prefill(t, wl.chunk, want_out=False, check_state=(t + wl.chunk >= wl.tokens))
+        t += wl.chunk
+    for sidx in range(wl.decode_steps):
+        ls.decode(sidx)
+    summ = ls.summary()
+    print("cfg3 sample", summ)
+    assert summ["resyncs"] <= 2, summ
 
 
 def test_bf16_generic_kernels_flag():
