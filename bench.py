@@ -318,7 +318,7 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
     dev = torch.device(f"cuda:{local_rank}")
     inputs = WorkloadInputs(wl.with_(batch=wl.batch * world))
     rows = rank_rows(rank, wl.batch)
-    B, C, S = wl.batch, wl.chunk, wl.decode_steps
+    B, C, S = wl.batch, wl.chunk, (args.decode_steps or wl.decode_steps)
     T = args.decode_prefill if args.decode_prefill else wl.tokens
     tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window, wl.sparse, C,
@@ -476,6 +476,7 @@ def main():
     ap.add_argument("--workload", default="default", choices=["default", "cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--decode-prefill", type=int, default=0, help="tokens of the untimed prefill of cfg3 (0 = full)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="decode calls per step of cfg3 (0 = the workload's 256)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="default line without the cfg3 entry")
     args = ap.parse_args()

@@ -4,11 +4,12 @@
 // computed on the way:
 //
 //   rows of the stream = sparse-cache slots 0..lambda-1, then the window ring slots 0..eta-1, in
-//   tiles of 128 rows.  Per tile (one thread per row, two row groups of 128 threads work on
-//   alternate tiles so that one group's arithmetic overlaps the other's loads and MMAs):
-//     [U | Z] = K_tile [W | Q^T]          tcgen05.mma  M=128, N=80, K=d   (pre-activations, q.k)
-//     phi = feature map of U, rounded to bf16; den = phi . s
-//     P = phi H                            tcgen05.mma  M=128, N=d,  K=128
+//   tiles of 128 rows.  Two row groups of 256 threads work on alternate tiles (two threads per row:
+//   one per half of the feature map / half of the value columns), so that one group's arithmetic
+//   overlaps the other's loads and MMAs.  Per tile:
+//     [U | Z] = K_tile [W | Q^T]          tcgen05.mma  M=128, N=80,   K=d   (pre-activations, q.k)
+//     phi = feature map of U, rounded to bf16
+//     [P | den] = phi [H | s_hi s_lo]      tcgen05.mma  M=128, N=d+16, K=128 (s split in two bf16 parts)
 //     score = || P / den - v ||            for sparse-cache rows and the evicted pair (Eq. 10)
 //     O^T += V_tile^T Pr^T                 tcgen05.mma  M=d(128), N=16, K=128 (Eq. 14 numerator),
 //                                          Pr = exp(z - m) with a running maximum per query row
@@ -30,7 +31,7 @@ namespace lola {
 
 constexpr int kDecQ = 8;          // query rows per unit the kernel carries (group size g <= 8)
 constexpr int kDecMaxTiles = 16;  // (lambda + eta rounded up to 64) / 128 <= 16
-constexpr int kDecThreads = 256;
+constexpr int kDecThreads = 512;  // two row groups of 256
 
 template <int DPL>
 struct DecodeSmem {
@@ -38,21 +39,21 @@ struct DecodeSmem {
   static constexpr int kblk = d / 64;
   static constexpr uint32_t b1_blk = 80 * 128;                       // one K block of [W^T ; Q]: 80 rows
   static constexpr uint32_t b1 = 0;                                  // [kblk][80][128B]
-  static constexpr uint32_t hmn = 2 * b1_blk;                        // H, MN-major: [kblk (c blocks)][128 j][128B]
-  static constexpr uint32_t phiq = hmn + 2 * 16384;                  // phi(Q), K-major: [2 j blocks][16][128B]
+  static constexpr uint32_t ht_blk = (d + 16) * 128;                 // one j block of [H^T ; s_hi ; s_lo ; ...]
+  static constexpr uint32_t ht = 2 * b1_blk;                         // K-major: [2 j blocks][d + 16 rows][128B]
+  static constexpr uint32_t phiq = ht + 2 * (128 + 16) * 128;        // phi(Q), K-major: [2 j blocks][16][128B]
   static constexpr uint32_t stage0 = phiq + 4096;
   static constexpr uint32_t st_k = 0;                                // K tile [kblk][128][128B]; then phi tile [2][128][128B]
-  static constexpr uint32_t st_v = 32768;                            // V tile [kblk][128 keys][128B]
+  static constexpr uint32_t st_v = 32768;                            // V tile [kblk][128 keys][128B]; at the end O^T partials
   static constexpr uint32_t st_pt = 65536;                           // Pr^T, K-major: [2 key blocks][16][128B]
   static constexpr uint32_t stage_bytes = 65536 + 4096;
   static constexpr uint32_t misc = stage0 + 2 * stage_bytes;         // small arrays, see DecodeMisc
-  static constexpr uint32_t total = misc + 32768;
+  static constexpr uint32_t total = misc + 28672;
   static constexpr uint32_t bytes = total + 1024;                    // slack to align the base to 1024
 };
 
-// small shared arrays (all fp32 / int unless noted)
+// small shared arrays
 struct DecodeMisc {
-  float s_vec[128];
   float qf[kDecQ][128];          // query rows, fp32
   float phiq_f[kDecQ][128];      // phi(q) rounded to bf16, as fp32
   float u_s[kDecQ][64];
@@ -61,9 +62,9 @@ struct DecodeMisc {
   float redmax[2][4][kDecQ];
   unsigned long long redkey[2][4];
   float red12[2][4][2];
+  float ssp[2][128];             // partial squared errors of the second half of the value columns
   float wg_m[2][kDecQ];
-  float wg_l[2][4][kDecQ];
-  float opart[2][128][kDecQ];
+  float wg_l[2][8][kDecQ];
   // per-tile list of the rows left out of O^T
   unsigned long long cand_key[kDecMaxTiles];
   float cand_score[kDecMaxTiles], cand_min2[kDecMaxTiles];
@@ -74,13 +75,21 @@ struct DecodeMisc {
   uint64_t bars[8];
   uint32_t tmem_slot;
 };
-static_assert(sizeof(DecodeMisc) <= 32768, "misc region too small");
+static_assert(sizeof(DecodeMisc) <= 28672, "misc region too small");
 
 __device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long x, int o) {
   unsigned lo = __shfl_xor_sync(0xffffffffu, (unsigned)x, o);
   unsigned hi = __shfl_xor_sync(0xffffffffu, (unsigned)(x >> 32), o);
   return ((unsigned long long)hi << 32) | lo;
 }
+
+// two fp32 -> packed bf16x2 (a in the low half), and the rounded values back as fp32 by bit moves
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ float bf16lo_f(uint32_t p) { return __uint_as_float(p << 16); }
+__device__ __forceinline__ float bf16hi_f(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
 
 // Loads of one tile: two half tiles of 64 rows; a half tile is a block of sparse-cache slots, a block
 // of ring slots, or nothing (a box that lies entirely outside the ring tensor reads as zeros).
@@ -109,6 +118,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
   constexpr int F = 64, D = 128;
+  constexpr int HC = d / 2;                  // value columns per thread of a row pair
   constexpr float kLog2e = 1.4426950408889634f;
   typedef __nv_bfloat16 T;
   extern __shared__ uint8_t smem_raw[];
@@ -117,49 +127,70 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   DecodeMisc& X = *reinterpret_cast<DecodeMisc*>(sm + S::misc);
 
   const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
-  const int tid = threadIdx.x, wg = tid >> 7, t = tid & 127, warp = tid >> 5, wq = warp & 3, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int wg = tid >> 8;                   // row group
+  const int wq = warp & 3;                   // tensor-memory lane quadrant of this warp
+  const int hf = (warp >> 2) & 1;            // which half of the row's work this thread does
+  const int t = wq * 32 + lane;              // row of the tile = tensor-memory lane
+  const bool lead = (tid & 255) == 0;        // issues the row group's TMA and MMAs
   const int lam = L.lam, eta = L.eta, g = L.g;
   const int nGB = lam / 64, nRB = (eta + 63) / 64, NT = (nGB + nRB + 1) / 2;
-  const int s_ev = c.n_seen % eta;          // ring slot of the pair that leaves = slot the new pair takes
+  const int s_ev = c.n_seen % eta;           // ring slot of the pair that leaves = slot the new pair takes
   const int pos_ev = c.n_seen - eta;
+  const float sl2 = L.scale * kLog2e;        // q.k in log2 units
   float* scu = L.score + (size_t)unit * (lam + L.cmax);
 
-  const uint32_t bar_k = sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + (uint32_t)wg * 24u;
-  const uint32_t bar_v = bar_k + 8, bar_mma = bar_k + 16;
+  const uint32_t bar_k = sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + (uint32_t)wg * 32u;
+  const uint32_t bar_v = bar_k + 8, bar_mma = bar_k + 16, bar_mma3 = bar_k + 24;
   const uint32_t stage = sbase + S::stage0 + (uint32_t)wg * S::stage_bytes;
   uint8_t* stage_p = sm + S::stage0 + (size_t)wg * S::stage_bytes;
-  uint32_t pk = 0, pv = 0, pm = 0;
+  uint32_t pk = 0, pv = 0, pm = 0, pm3 = 0;
   bool ok = true;
 
   if (tid == 0) {
-    for (int i = 0; i < 6; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + 8u * i, 1);
+    for (int i = 0; i < 8; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + 8u * i, 1);
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
   __syncthreads();
   // first tile of each row group starts to stream while the operands below are prepared
-  if (t == 0 && wg < NT) {
+  if (lead && wg < NT) {
     decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, wg, nGB, nRB, unit, bar_k);
     decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, wg, nGB, nRB, unit, bar_v);
   }
 
   // ---- operands that stay for the whole unit
   {
-    // H (fp32, [D][d]) -> bf16, MN-major: c block, row j, 64 c per 128-byte row
-    const float4* Hg = reinterpret_cast<const float4*>(L.H + (size_t)unit * D * d);
-    constexpr int per_row = d / 8;
-#pragma unroll 4
-    for (int i = tid; i < D * per_row; i += kDecThreads) {
-      const int j = i / per_row, c8 = (i % per_row) * 8;
-      float4 a = Hg[(size_t)i * 2], bq = Hg[(size_t)i * 2 + 1];
-      float f8[8] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w};
-      *reinterpret_cast<uint4*>(sm + S::hmn + (c8 >> 6) * 16384 + tc::sw128_off(j, (c8 & 63) >> 3)) = tc::pack8_bf16(f8);
+    // H (fp32 [D][d]) -> bf16 H^T, K-major: row c, 64 j per 128-byte row, two j blocks.  A thread
+    // gathers 8 consecutive j of one column c (each load coalesced over the warp's 32 columns).
+    const float* Hg = L.H + (size_t)unit * D * d;
+    for (int i = tid; i < d * (D / 8); i += kDecThreads) {
+      const int cc = i % d, jc = i / d;
+      float f8[8];
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) f8[jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
+    }
+    // rows d, d+1: s as the sum of two bf16 parts (phi . s_hi + phi . s_lo keeps the fp32 normaliser)
+    if (tid < D) {
+      const float sv = L.s[(size_t)unit * D + tid];
+      const __nv_bfloat16 hi = __float2bfloat16_rn(sv);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(sv - __bfloat162float(hi));
+      const int ch = (tid & 63) >> 3;
+      *reinterpret_cast<T*>(sm + S::ht + (tid >> 6) * S::ht_blk + tc::sw128_off(d, ch) + (tid & 7) * 2) = hi;
+      *reinterpret_cast<T*>(sm + S::ht + (tid >> 6) * S::ht_blk + tc::sw128_off(d + 1, ch) + (tid & 7) * 2) = lo;
+    }
+    // rows d+2 .. d+15 of both j blocks: zero
+    for (int i = tid; i < 2 * 14 * 8; i += kDecThreads) {
+      const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
+      *reinterpret_cast<uint4*>(sm + S::ht + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
     }
     // W^T image (prepared once per layer in the operand layout): rows 0..63 of each K block of B1
     const uint4* img = wt_image + (size_t)h * kblk * 512;
     for (int i = tid; i < kblk * 512; i += kDecThreads)
       *reinterpret_cast<uint4*>(sm + S::b1 + (i >> 9) * S::b1_blk + (i & 511) * 16) = img[i];
     // query rows: B1 rows 64..79 (rows >= g are zero) and an fp32 copy
+    constexpr int per_row = d / 8;
     for (int i = tid; i < 16 * per_row; i += kDecThreads) {
       const int r = i / per_row, ch = i % per_row;
       uint4 val = make_uint4(0, 0, 0, 0);
@@ -175,7 +206,6 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
         }
       }
     }
-    if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
     if (tid < d) {
       X.knew[tid] = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + tid);
       X.vnew[tid] = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + tid);
@@ -189,11 +219,10 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     }
   }
   __syncthreads();
-  // u = q W on the CUDA cores (g rows only) from the W^T operand image, then phi(q), its normaliser
-  // and q . k_new
+  // u = q W on the CUDA cores (g rows only) from the W^T operand image
   for (int i = tid; i < g * F; i += kDecThreads) {
     const int r = i >> 6, f = i & 63;
-    float a = 0.f;
+    float a0 = 0.f, a1 = 0.f;
 #pragma unroll
     for (int ch = 0; ch < d / 8; ++ch) {
       uint4 raw = *reinterpret_cast<const uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(f, ch & 7));
@@ -201,13 +230,14 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         float2 ww = __bfloat1622float2(w2[q]);
-        a = fmaf(X.qf[r][ch * 8 + 2 * q], ww.x, a);
-        a = fmaf(X.qf[r][ch * 8 + 2 * q + 1], ww.y, a);
+        a0 = fmaf(X.qf[r][ch * 8 + 2 * q], ww.x, a0);
+        a1 = fmaf(X.qf[r][ch * 8 + 2 * q + 1], ww.y, a1);
       }
     }
-    X.u_s[r][f] = a;
+    X.u_s[r][f] = a0 + a1;
   }
   __syncthreads();
+  // phi(q), its normaliser phi(q) . s and q . k_new
   if (warp < g) {
     const int r = warp;
     float u0 = X.u_s[r][lane], u1 = X.u_s[r][lane + 32];
@@ -228,13 +258,13 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       const int j = js[q];
       X.phiq_f[r][j] = vals[q];
       *reinterpret_cast<T*>(sm + S::phiq + (j >> 6) * 2048 + tc::sw128_off(r, (j & 63) >> 3) + (j & 7) * 2) = __float2bfloat16_rn(vals[q]);
-      ld = fmaf(vals[q], X.s_vec[j], ld);
+      ld = fmaf(vals[q], L.s[(size_t)unit * D + j], ld);
     }
     ld = warp_sum(ld);
     float zz = 0.f;
     for (int j = lane; j < d; j += 32) zz = fmaf(X.qf[r][j], X.knew[j], zz);
     zz = warp_sum(zz);
-    if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * L.scale; }
+    if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * sl2; }
   }
   tc::fence_async_smem();
   tc::fence_before_sync();
@@ -242,24 +272,26 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   tc::fence_after_sync();
   const uint32_t tmem = X.tmem_slot;
   const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-  const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // [U | Z], then P
+  const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // [U | Z], then [P | den]
   const uint32_t tm_o = tm_a + 160u;                            // O^T: lanes = value column, 16 columns = query rows
   const uint32_t idesc1 = tc::make_idesc_bf16(128, 80, false, false);
-  const uint32_t idesc2 = tc::make_idesc_bf16(128, d, false, true);
+  const uint32_t idesc2 = tc::make_idesc_bf16(128, d + 16, false, false);
+  const uint32_t idesc0 = tc::make_idesc_bf16(128, 16, false, false);
   const uint32_t idesc3 = tc::make_idesc_bf16(128, 16, true, false);
 
   bool have_o = false;
   if (wg == 0) {
     // O^T = H^T phi(Q)^T: the linear term enters the running sums with weight exp(0 - m), m = 0 so far
-    if (t == 0) {
+    if (lead) {
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::hmn + ks * 2048, 16384, 1024),
-                        tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc3, ks > 0);
+        tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
+                        tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc0, ks > 0);
     }
     have_o = true;
   }
 
+  // running maxima (log2 units, uniform over the row group) and this thread's share of the sums
   float m_run[kDecQ], lpart[kDecQ];
 #pragma unroll
   for (int r = 0; r < kDecQ; ++r) { m_run[r] = 0.f; lpart[r] = 0.f; }
@@ -275,7 +307,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     // ---- [U | Z] = K_tile [W | Q^T]
     ok = tc::mbar_wait(bar_k, pk) && ok; pk ^= 1;
     tc::fence_after_sync();
-    if (t == 0) {
+    if (lead) {
 #pragma unroll
       for (int ks = 0; ks < d / 16; ++ks)
         tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
@@ -286,77 +318,70 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     tc::fence_after_sync();
 
     float z[kDecQ];
-    float den = 0.f;
     {
       float zraw[8];
       tc::tmem_ld8(tm_a + lane_addr + 64, zraw);
 #pragma unroll
-      for (int r = 0; r < kDecQ; ++r) z[r] = valid ? zraw[r] * L.scale : -CUDART_INF_F;
-      float u0[32], u1[32];
-      tc::tmem_ld32(tm_a + lane_addr, u0);
-      tc::tmem_ld32(tm_a + lane_addr + 32, u1);
-      // feature map, one half at a time; each half goes to the A operand of the second product
-      // (over the key tile, which the first product no longer needs)
-      float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+      for (int r = 0; r < kDecQ; ++r) z[r] = valid ? zraw[r] * sl2 : -CUDART_INF_F;
+      if (hf == 0) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        mx = fmaxf(mx, fmaxf(u0[i], u1[i]));
-        mn = fminf(mn, fminf(u0[i], u1[i]));
+        for (int r = 0; r < kDecQ; ++r) {
+          float wm = warp_max(z[r]);
+          if (lane == 0) X.redmax[wg][wq][r] = wm;
+        }
+      }
+      // this thread's half of the feature map: hf = 0: softmax(u), hf = 1: softmax(-u); in place
+      float e[64];
+      tc::tmem_ld64(tm_a + lane_addr, e);
+      const float sgn = hf ? -kLog2e : kLog2e;
+      if (L.phi_kind == 1) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
+      } else {
+        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
+#pragma unroll
+        for (int i = 0; i < 64; i += 4) {
+          m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn);
+          m2 = fmaxf(m2, e[i + 2] * sgn); m3 = fmaxf(m3, e[i + 3] * sgn);
+        }
+        const float mm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 64; i += 4) {
+          e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
+          e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
+          e[i + 2] = tc::fast_exp2(fmaf(e[i + 2], sgn, -mm)); s2 += e[i + 2];
+          e[i + 3] = tc::fast_exp2(fmaf(e[i + 3], sgn, -mm)); s3 += e[i + 3];
+        }
+        const float inv = 1.0f / ((s0 + s1) + (s2 + s3));
+#pragma unroll
+        for (int i = 0; i < 64; ++i) e[i] *= inv;
       }
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float f[64];
-        if (L.phi_kind == 1) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            f[i] = expf(half ? -u0[i] : u0[i]);
-            f[32 + i] = expf(half ? -u1[i] : u1[i]);
-          }
-        } else {
-          const float off = half ? mn : -mx;
-          float ssum = 0.f;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            f[i] = tc::fast_exp2(((half ? -u0[i] : u0[i]) + off) * kLog2e);
-            f[32 + i] = tc::fast_exp2(((half ? -u1[i] : u1[i]) + off) * kLog2e);
-          }
-#pragma unroll
-          for (int i = 0; i < 64; ++i) ssum += f[i];
-          const float inv = 1.0f / ssum;
-#pragma unroll
-          for (int i = 0; i < 64; ++i) f[i] *= inv;
-        }
-#pragma unroll
-        for (int i = 0; i < 64; ++i) {
-          f[i] = round_bf16f(f[i]);
-          den = fmaf(f[i], X.s_vec[half * 64 + i], den);
-        }
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-          *reinterpret_cast<uint4*>(stage_p + S::st_k + half * 16384 + tc::sw128_off(t, ch)) = tc::pack8_bf16(f + ch * 8);
+      for (int ch = 0; ch < 8; ++ch) {
+        uint4 o;
+        o.x = pack_bf16x2(e[ch * 8], e[ch * 8 + 1]);
+        o.y = pack_bf16x2(e[ch * 8 + 2], e[ch * 8 + 3]);
+        o.z = pack_bf16x2(e[ch * 8 + 4], e[ch * 8 + 5]);
+        o.w = pack_bf16x2(e[ch * 8 + 6], e[ch * 8 + 7]);
+        *reinterpret_cast<uint4*>(stage_p + S::st_k + hf * 16384 + tc::sw128_off(t, ch)) = o;
       }
     }
     tc::fence_async_smem();
     tc::fence_before_sync();
-    tc::named_bar_sync(1 + wg, 128);
+    tc::named_bar_sync(1 + wg, 256);
     tc::fence_after_sync();
-    // ---- P = phi H
-    if (t == 0) {
+    // ---- [P | den] = phi [H | s_hi s_lo]
+    if (lead) {
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks)
         tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                        tc::make_desc_sw128(sbase + S::hmn + ks * 2048, 16384, 1024), idesc2, ks > 0);
+                        tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024), idesc2, ks > 0);
       tc::mma_commit(bar_mma);
     }
-    // meanwhile: running maximum of q.k per query row (every valid row counts, also the one that will
-    // be folded: any m >= the true maximum leaves Eq. 14 unchanged)
+    // running maximum of q.k per query row (every valid row counts, also the one that will be folded:
+    // any m >= the true maximum leaves Eq. 14 unchanged)
     float m_new[kDecQ];
-#pragma unroll
-    for (int r = 0; r < kDecQ; ++r) {
-      float wm = warp_max(z[r]);
-      if (lane == 0) X.redmax[wg][wq][r] = wm;
-    }
-    tc::named_bar_sync(1 + wg, 128);
 #pragma unroll
     for (int r = 0; r < kDecQ; ++r)
       m_new[r] = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[wg][0][r], X.redmax[wg][1][r])),
@@ -365,37 +390,40 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     ok = tc::mbar_wait(bar_v, pv) && ok; pv ^= 1;
     ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
     tc::fence_after_sync();
-    // ---- Eq. 10
+    // ---- Eq. 10: this thread's half of the value columns
     float score;
     {
-      float ss = 0.f;
-      const bool pos_den = den > 0.f;
+      float dn[2];
+      tc::tmem_ld2(tm_a + lane_addr + d, dn);
+      const float den = dn[0] + dn[1];
+      const float inv = den > 0.f ? 1.0f / den : 0.f;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-      for (int c0 = 0; c0 < d; c0 += 32) {
+      for (int c0 = 0; c0 < HC; c0 += 32) {
         float p[32];
-        tc::tmem_ld32(tm_a + lane_addr + c0, p);
+        tc::tmem_ld32(tm_a + lane_addr + hf * HC + c0, p);
 #pragma unroll
         for (int q8 = 0; q8 < 4; ++q8) {
-          const int cc = c0 + q8 * 8;
+          const int cc = hf * HC + c0 + q8 * 8;
           uint4 raw = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (cc >> 6) * 16384 + tc::sw128_off(t, (cc & 63) >> 3));
-          const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            float2 vv = __bfloat1622float2(v2[q]);
-            float d0 = (pos_den ? p[q8 * 8 + 2 * q] / den : 0.f) - vv.x;
-            float d1 = (pos_den ? p[q8 * 8 + 2 * q + 1] / den : 0.f) - vv.y;
-            ss = fmaf(d0, d0, ss);
-            ss = fmaf(d1, d1, ss);
-          }
+          float d0 = fmaf(p[q8 * 8 + 0], inv, -bf16lo_f(raw.x)), d1 = fmaf(p[q8 * 8 + 1], inv, -bf16hi_f(raw.x));
+          float d2 = fmaf(p[q8 * 8 + 2], inv, -bf16lo_f(raw.y)), d3 = fmaf(p[q8 * 8 + 3], inv, -bf16hi_f(raw.y));
+          float d4 = fmaf(p[q8 * 8 + 4], inv, -bf16lo_f(raw.z)), d5 = fmaf(p[q8 * 8 + 5], inv, -bf16hi_f(raw.z));
+          float d6 = fmaf(p[q8 * 8 + 6], inv, -bf16lo_f(raw.w)), d7 = fmaf(p[q8 * 8 + 7], inv, -bf16hi_f(raw.w));
+          a0 = fmaf(d0, d0, a0); a1 = fmaf(d1, d1, a1); a2 = fmaf(d2, d2, a2); a3 = fmaf(d3, d3, a3);
+          a0 = fmaf(d4, d4, a0); a1 = fmaf(d5, d5, a1); a2 = fmaf(d6, d6, a2); a3 = fmaf(d7, d7, a3);
         }
       }
-      score = sqrtf(ss);
+      const float ss = (a0 + a1) + (a2 + a3);
+      if (hf == 1) X.ssp[wg][t] = ss;
+      tc::named_bar_sync(1 + wg, 256);
+      score = sqrtf(ss + X.ssp[wg][t]);       // hf = 1 threads double their own half; they do not use the score
     }
-    if (scored && ok) scu[is_g ? R : lam] = score;
     // lowest score of the tile (ties: the younger pair), and the two lowest values
-    unsigned long long key = scored ? (((unsigned long long)__float_as_uint(score) << 32) | (unsigned)(0x7fffffff - pos))
-                                    : ~0ull;
-    {
+    unsigned long long key = ~0ull;
+    if (hf == 0) {
+      if (scored && ok) scu[is_g ? R : lam] = score;
+      if (scored) key = ((unsigned long long)__float_as_uint(score) << 32) | (unsigned)(0x7fffffff - pos);
       unsigned long long k = key;
       float a1 = scored ? score : CUDART_INF_F, a2 = CUDART_INF_F;
 #pragma unroll
@@ -409,48 +437,60 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       }
       if (lane == 0) { X.redkey[wg][wq] = k; X.red12[wg][wq][0] = a1; X.red12[wg][wq][1] = a2; }
     }
-    tc::named_bar_sync(1 + wg, 128);
+    tc::named_bar_sync(1 + wg, 256);
     unsigned long long tkey = X.redkey[wg][0];
 #pragma unroll
     for (int w = 1; w < 4; ++w) tkey = X.redkey[wg][w] < tkey ? X.redkey[wg][w] : tkey;
-    const bool left_out = scored && key == tkey;
+    // the row left out of O^T: both threads of the row know it from the row's position
+    const unsigned long long rowkey_lo = (unsigned)(0x7fffffff - pos);
+    const bool left_out = scored && (unsigned)tkey == (unsigned)rowkey_lo && tkey != ~0ull;
     if (left_out) {
-      float a1 = X.red12[wg][0][0], a2 = X.red12[wg][0][1];
+      if (hf == 0) {
+        float a1 = X.red12[wg][0][0], a2 = X.red12[wg][0][1];
 #pragma unroll
-      for (int w = 1; w < 4; ++w) {
-        float b1 = X.red12[wg][w][0], b2 = X.red12[wg][w][1];
-        float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
-        a2 = fminf(hi, fminf(a2, b2));
-        a1 = lo;
-      }
-      X.cand_key[tile] = key;
-      X.cand_score[tile] = score;
-      X.cand_min2[tile] = a2;
-      X.cand_row[tile] = R;
+        for (int w = 1; w < 4; ++w) {
+          float b1 = X.red12[wg][w][0], b2 = X.red12[wg][w][1];
+          float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
+          a2 = fminf(hi, fminf(a2, b2));
+          a1 = lo;
+        }
+        X.cand_key[tile] = key;
+        X.cand_score[tile] = score;
+        X.cand_min2[tile] = a2;
+        X.cand_row[tile] = R;
 #pragma unroll
-      for (int r = 0; r < kDecQ; ++r) X.cand_z[tile][r] = z[r];
+        for (int r = 0; r < kDecQ; ++r) X.cand_z[tile][r] = z[r];
 #pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        X.cand_phi[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_k + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
-        if (ch < d / 8)
+        for (int ch = 0; ch < 16; ++ch)
+          X.cand_phi[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_k + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
+      } else {
+#pragma unroll
+        for (int ch = 0; ch < d / 8; ++ch)
           X.cand_v[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
       }
     }
-    // ---- softmax weights of the tile (bf16, the sums use the rounded weights) and running sums
+    // ---- softmax weights of the tile (bf16; the sums use the rounded weights): query rows 4 hf .. 4 hf + 3
     {
       bool moved = false;
       float alpha[kDecQ];
 #pragma unroll
       for (int r = 0; r < kDecQ; ++r) {
-        alpha[r] = tc::fast_exp2((m_run[r] - m_new[r]) * kLog2e);
+        alpha[r] = tc::fast_exp2(m_run[r] - m_new[r]);
         moved = moved || (m_new[r] != m_run[r]);
-        float p = (valid && !left_out) ? tc::fast_exp2((z[r] - m_new[r]) * kLog2e) : 0.f;
-        p = round_bf16f(p);
-        lpart[r] = lpart[r] * alpha[r] + p;
+        lpart[r] *= alpha[r];
         m_run[r] = m_new[r];
-        *reinterpret_cast<T*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = __float2bfloat16_rn(p);
       }
-      if (have_o && moved) {                     // uniform over the row group
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) {
+        const int r = hf * 4 + rr;
+        if (r < kDecQ) {
+          float p = (valid && !left_out) ? tc::fast_exp2(z[r] - m_new[r]) : 0.f;
+          const __nv_bfloat16 pb = __float2bfloat16_rn(p);
+          lpart[r] += __bfloat162float(pb);
+          *reinterpret_cast<T*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = pb;
+        }
+      }
+      if (have_o && moved && hf == 0) {          // `moved` is uniform over the row group
         float ov[8];
         tc::tmem_ld8(tm_o + lane_addr, ov);
 #pragma unroll
@@ -460,40 +500,45 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     }
     tc::fence_async_smem();
     tc::fence_before_sync();
-    tc::named_bar_sync(1 + wg, 128);
+    tc::named_bar_sync(1 + wg, 256);
     tc::fence_after_sync();
     // ---- O^T += V^T Pr^T; the key/phi buffer is free for the next tile of this row group
-    if (t == 0) {
+    if (lead) {
       if (tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
         tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(stage + S::st_v + ks * 2048, 16384, 1024),
                         tc::make_desc_sw128(stage + S::st_pt + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc3,
                         (have_o || ks > 0) ? 1u : 0u);
-      tc::mma_commit(bar_mma);
+      tc::mma_commit(bar_mma3);
+      // the value buffer is free once this product is done; everybody else meets the leader again at
+      // the next barrier, before anything of this product's operands or O^T is touched
+      ok = tc::mbar_wait(bar_mma3, pm3) && ok;
+      tc::fence_after_sync();
+      if (tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_v);
     }
+    pm3 ^= 1;
     have_o = true;
-    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
-    tc::fence_after_sync();
-    if (t == 0 && tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_v);
   }
 
-  // ---- per row group: maximum, sums, partial O^T
+  // ---- per row group: maximum, sums, partial O^T (kept in the group's own value buffer)
+  tc::fence_before_sync();
+  tc::named_bar_sync(1 + wg, 256);              // the leader has seen the last O^T product complete
+  tc::fence_after_sync();
 #pragma unroll
   for (int r = 0; r < kDecQ; ++r) {
     float ls = warp_sum(lpart[r]);
-    if (lane == 0) X.wg_l[wg][wq][r] = ls;
+    if (lane == 0) X.wg_l[wg][warp & 7][r] = ls;
+    if (t == r && hf == 0) X.wg_m[wg][r] = m_run[r];
   }
-#pragma unroll
-  for (int r = 0; r < kDecQ; ++r)
-    if (t == r) X.wg_m[wg][r] = m_run[r];          // m_run is uniform over the row group
-  {
+  float* opart = reinterpret_cast<float*>(stage_p + S::st_v);   // [128][kDecQ]
+  if (hf == 0) {
     float ov[8];
 #pragma unroll
     for (int r = 0; r < kDecQ; ++r) ov[r] = 0.f;
     if (have_o) tc::tmem_ld8(tm_o + lane_addr, ov);
 #pragma unroll
-    for (int r = 0; r < kDecQ; ++r) X.opart[wg][t][r] = ov[r];
+    for (int r = 0; r < kDecQ; ++r) opart[t * kDecQ + r] = ov[r];
   }
   tc::fence_before_sync();
   __syncthreads();
@@ -517,28 +562,30 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
   const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
 
-  // ---- Eq. 14
-  if (tid < d && ok) {
-    const int cc = tid;
-    for (int r = 0; r < g; ++r) {
+  // ---- Eq. 14: thread (query row r, value column cc)
+  if (ok) {
+    const float* op0 = reinterpret_cast<const float*>(sm + S::stage0 + S::st_v);
+    const float* op1 = reinterpret_cast<const float*>(sm + S::stage0 + S::stage_bytes + S::st_v);
+    for (int i = tid; i < g * d; i += kDecThreads) {
+      const int r = i / d, cc = i % d;
       const float m0 = X.wg_m[0][r], m1 = X.wg_m[1][r];
       const float mf = fmaxf(fmaxf(m0, m1), X.zn[r]);
-      const float a0 = tc::fast_exp2((m0 - mf) * kLog2e), a1 = tc::fast_exp2((m1 - mf) * kLog2e);
+      const float a0 = tc::fast_exp2(m0 - mf), a1 = tc::fast_exp2(m1 - mf);
       float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-      for (int w = 0; w < 4; ++w) { l0 += X.wg_l[0][w][r]; l1 += X.wg_l[1][w][r]; }
-      float num = a0 * X.opart[0][cc][r] + a1 * X.opart[1][cc][r];
+      for (int w = 0; w < 8; ++w) { l0 += X.wg_l[0][w][r]; l1 += X.wg_l[1][w][r]; }
+      float num = a0 * op0[cc * kDecQ + r] + a1 * op1[cc * kDecQ + r];
       float den = a0 * l0 + a1 * l1;
-      for (int i = 0; i < NT; ++i) {
-        if (i == lt || X.cand_key[i] == ~0ull) continue;
-        const float p = round_bf16f(tc::fast_exp2((X.cand_z[i][r] - mf) * kLog2e));
-        num = fmaf(p, __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[i][0])[cc]), num);
+      for (int ti = 0; ti < NT; ++ti) {
+        if (ti == lt || X.cand_key[ti] == ~0ull) continue;
+        const float p = round_bf16f(tc::fast_exp2(X.cand_z[ti][r] - mf));
+        num = fmaf(p, __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[ti][0])[cc]), num);
         den += p;
       }
-      const float pn = tc::fast_exp2((X.zn[r] - mf) * kLog2e);
+      const float pn = tc::fast_exp2(X.zn[r] - mf);
       num = fmaf(pn, X.vnew[cc], num);
       den += pn;
-      const float e = tc::fast_exp2(-mf * kLog2e);
+      const float e = tc::fast_exp2(-mf);
       num = fmaf(e * X.dotL[r], __bfloat162float(vL[cc]), num);
       den = fmaf(e, X.lden[r] + X.dotL[r], den);
       ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
@@ -599,7 +646,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
     }
   }
-  if (!ok && t == 0) atomicOr(L.status, 8);
+  if (!ok && (tid & 255) == 0) atomicOr(L.status, 8);
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tmem, 512);
