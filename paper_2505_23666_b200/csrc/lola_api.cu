@@ -230,8 +230,12 @@ template <int DPL>
 int launch_decode_fused(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   LaunchScope scope(st, LOLA_KERNEL_DECODE, s);
-  k_decode_tc<DPL><<<L.B * L.Hkv, kDecThreads, DecodeSmem<DPL>::bytes, s>>>(
-      L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, (const uint4*)(st->base + st->lay.wt));
+  if (L.g <= 4)
+    k_decode_tc<DPL, 4><<<L.B * L.Hkv, kDecThreads, DecodeSmem<DPL>::bytes, s>>>(
+        L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, (const uint4*)(st->base + st->lay.wt));
+  else
+    k_decode_tc<DPL, 8><<<L.B * L.Hkv, kDecThreads, DecodeSmem<DPL>::bytes, s>>>(
+        L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, (const uint4*)(st->base + st->lay.wt));
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
@@ -323,10 +327,15 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
               make_rows_map(&st->tm_gv, L.gv, U, cfg->sparse, cfg->head_dim, 64) &&
               make_rows_map(&st->tm_wk, L.wk, U, cfg->window, cfg->head_dim, 64) &&
               make_rows_map(&st->tm_wv, L.wv, U, cfg->window, cfg->head_dim, 64);
-    cudaError_t e = cfg->head_dim == 128
-        ? cudaFuncSetAttribute(k_decode_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes)
-        : cudaFuncSetAttribute(k_decode_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
-    if (!ok || e != cudaSuccess) st->fused_decode = false;   // the kernel chain serves every shape
+    cudaError_t e = cudaSuccess, e2 = cudaSuccess;
+    if (cfg->head_dim == 128) {
+      e = cudaFuncSetAttribute(k_decode_tc<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
+      e2 = cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
+    } else {
+      e = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+      e2 = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+    }
+    if (!ok || e != cudaSuccess || e2 != cudaSuccess) st->fused_decode = false;   // the kernel chain serves every shape
   }
   if (rc == LOLA_OK && st->tensor_path) {
     cudaStream_t s = (cudaStream_t)stream;

@@ -43,7 +43,7 @@ struct DecodeSmem {
   static constexpr uint32_t ht = 2 * b1_blk;                         // K-major: [2 j blocks][d + 16 rows][128B]
   static constexpr uint32_t phiq = ht + 2 * (128 + 16) * 128;        // phi(Q), K-major: [2 j blocks][16][128B]
   static constexpr uint32_t stage0 = phiq + 4096;
-  static constexpr uint32_t st_k = 0;                                // K tile [kblk][128][128B]; then phi tile [2][128][128B]
+  static constexpr uint32_t st_k = 0;                                // K tile [kblk][128][128B]
   static constexpr uint32_t st_v = 32768;                            // V tile [kblk][128 keys][128B]; at the end O^T partials
   static constexpr uint32_t st_pt = 65536;                           // Pr^T, K-major: [2 key blocks][16][128B]
   static constexpr uint32_t stage_bytes = 65536 + 4096;
@@ -83,6 +83,11 @@ __device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long x,
   return ((unsigned long long)hi << 32) | lo;
 }
 
+// warp-wide maximum / minimum of fp32 values through the integer reduction instruction
+__device__ __forceinline__ int f2ord(float x) { int i = __float_as_int(x); return i ^ ((i >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+__device__ __forceinline__ float warp_max_redux(float x) { return ord2f(__reduce_max_sync(0xffffffffu, f2ord(x))); }
+
 // two fp32 -> packed bf16x2 (a in the low half), and the rounded values back as fp32 by bit moves
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
@@ -110,7 +115,7 @@ __device__ __forceinline__ void decode_issue_tile(uint32_t dst, const CUtensorMa
   }
 }
 
-template <int DPL>
+template <int DPL, int QR>
 __global__ void __launch_bounds__(kDecThreads, 1)
 k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image) {
@@ -160,16 +165,19 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   }
 
   // ---- operands that stay for the whole unit
+  constexpr int HI = d * (D / 8) / kDecThreads;
+  float hreg[HI][8];
+  const float* Hg = L.H + (size_t)unit * D * d;
   {
     // H (fp32 [D][d]) -> bf16 H^T, K-major: row c, 64 j per 128-byte row, two j blocks.  A thread
-    // gathers 8 consecutive j of one column c (each load coalesced over the warp's 32 columns).
-    const float* Hg = L.H + (size_t)unit * D * d;
-    for (int i = tid; i < d * (D / 8); i += kDecThreads) {
-      const int cc = i % d, jc = i / d;
-      float f8[8];
+    // gathers 8 consecutive j of one column c (each load coalesced over the warp's 32 columns).  All
+    // loads are issued here; they are converted and stored after the small query-side work below.
 #pragma unroll
-      for (int jj = 0; jj < 8; ++jj) f8[jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
-      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
+    for (int it = 0; it < HI; ++it) {
+      const int i = tid + it * kDecThreads;
+      const int cc = i % d, jc = i / d;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) hreg[it][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
     }
     // rows d, d+1: s as the sum of two bf16 parts (phi . s_hi + phi . s_lo keeps the fp32 normaliser)
     if (tid < D) {
@@ -196,7 +204,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       uint4 val = make_uint4(0, 0, 0, 0);
       if (r < g) val = *reinterpret_cast<const uint4*>((const T*)c.q + ((size_t)b * L.Hq + h * g + r) * d + ch * 8);
       *reinterpret_cast<uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(64 + r, ch & 7)) = val;
-      if (r < kDecQ) {
+      if (r < QR) {
         const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&val);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -266,6 +274,12 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     zz = warp_sum(zz);
     if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * sl2; }
   }
+#pragma unroll
+  for (int it = 0; it < HI; ++it) {
+    const int i = tid + it * kDecThreads;
+    const int cc = i % d, jc = i / d;
+    *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(hreg[it]);
+  }
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
@@ -274,6 +288,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
   const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // [U | Z], then [P | den]
   const uint32_t tm_o = tm_a + 160u;                            // O^T: lanes = value column, 16 columns = query rows
+  const uint32_t tm_phi = tm_a + 192u;                          // phi tile, bf16 pairs: 64 columns
   const uint32_t idesc1 = tc::make_idesc_bf16(128, 80, false, false);
   const uint32_t idesc2 = tc::make_idesc_bf16(128, d + 16, false, false);
   const uint32_t idesc0 = tc::make_idesc_bf16(128, 16, false, false);
@@ -292,9 +307,12 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   }
 
   // running maxima (log2 units, uniform over the row group) and this thread's share of the sums
-  float m_run[kDecQ], lpart[kDecQ];
+  // the two row groups take turns in the exponential-heavy feature-map phase (barriers 3 + wg):
+  // group 1 lets group 0 go first
+  if (wg == 1) asm volatile("bar.arrive 3, 512;" ::: "memory");
+  float m_run[QR], lpart[QR];
 #pragma unroll
-  for (int r = 0; r < kDecQ; ++r) { m_run[r] = 0.f; lpart[r] = 0.f; }
+  for (int r = 0; r < QR; ++r) { m_run[r] = 0.f; lpart[r] = 0.f; }
 
   for (int tile = wg; tile < NT; tile += 2) {
     const int R = tile * 128 + t;
@@ -317,20 +335,21 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
     tc::fence_after_sync();
 
-    float z[kDecQ];
+    float z[QR];
     {
       float zraw[8];
-      tc::tmem_ld8(tm_a + lane_addr + 64, zraw);
+      tc::tmem_ld8(tm_a + lane_addr + 64, zraw);   // 8 columns are loaded, the first QR are query rows
 #pragma unroll
-      for (int r = 0; r < kDecQ; ++r) z[r] = valid ? zraw[r] * sl2 : -CUDART_INF_F;
+      for (int r = 0; r < QR; ++r) z[r] = valid ? zraw[r] * sl2 : -CUDART_INF_F;
       if (hf == 0) {
 #pragma unroll
-        for (int r = 0; r < kDecQ; ++r) {
-          float wm = warp_max(z[r]);
+        for (int r = 0; r < QR; ++r) {
+          float wm = warp_max_redux(z[r]);
           if (lane == 0) X.redmax[wg][wq][r] = wm;
         }
       }
       // this thread's half of the feature map: hf = 0: softmax(u), hf = 1: softmax(-u); in place
+      tc::named_bar_sync(3 + wg, 512);
       float e[64];
       tc::tmem_ld64(tm_a + lane_addr, e);
       const float sgn = hf ? -kLog2e : kLog2e;
@@ -357,16 +376,15 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
 #pragma unroll
         for (int i = 0; i < 64; ++i) e[i] *= inv;
       }
+      // bf16 pairs into tensor memory: the A operand of the second product (K index = feature j)
+      uint32_t pk2[32];
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        uint4 o;
-        o.x = pack_bf16x2(e[ch * 8], e[ch * 8 + 1]);
-        o.y = pack_bf16x2(e[ch * 8 + 2], e[ch * 8 + 3]);
-        o.z = pack_bf16x2(e[ch * 8 + 4], e[ch * 8 + 5]);
-        o.w = pack_bf16x2(e[ch * 8 + 6], e[ch * 8 + 7]);
-        *reinterpret_cast<uint4*>(stage_p + S::st_k + hf * 16384 + tc::sw128_off(t, ch)) = o;
-      }
+      for (int i = 0; i < 32; ++i) pk2[i] = pack_bf16x2(e[2 * i], e[2 * i + 1]);
+      tc::tmem_st32u(tm_phi + lane_addr + hf * 32, pk2);
+      if (wg == 0) asm volatile("bar.arrive 4, 512;" ::: "memory"); else asm volatile("bar.arrive 3, 512;" ::: "memory");
     }
+    // the key tile is consumed: the next tile of this row group starts to stream now
+    if (lead && tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
     tc::fence_async_smem();
     tc::fence_before_sync();
     tc::named_bar_sync(1 + wg, 256);
@@ -375,15 +393,15 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     if (lead) {
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+        tc::mma_bf16_ts(tm_a, tm_phi + ks * 8,
                         tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024), idesc2, ks > 0);
       tc::mma_commit(bar_mma);
     }
     // running maximum of q.k per query row (every valid row counts, also the one that will be folded:
     // any m >= the true maximum leaves Eq. 14 unchanged)
-    float m_new[kDecQ];
+    float m_new[QR];
 #pragma unroll
-    for (int r = 0; r < kDecQ; ++r)
+    for (int r = 0; r < QR; ++r)
       m_new[r] = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[wg][0][r], X.redmax[wg][1][r])),
                        fmaxf(X.redmax[wg][2][r], X.redmax[wg][3][r]));
 
@@ -424,17 +442,16 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     if (hf == 0) {
       if (scored && ok) scu[is_g ? R : lam] = score;
       if (scored) key = ((unsigned long long)__float_as_uint(score) << 32) | (unsigned)(0x7fffffff - pos);
-      unsigned long long k = key;
-      float a1 = scored ? score : CUDART_INF_F, a2 = CUDART_INF_F;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        unsigned long long ko = shfl_xor_u64(k, o);
-        k = ko < k ? ko : k;
-        float b1 = __shfl_xor_sync(0xffffffffu, a1, o), b2 = __shfl_xor_sync(0xffffffffu, a2, o);
-        float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
-        a2 = fminf(hi, fminf(a2, b2));
-        a1 = lo;
-      }
+      // scores are norms (>= 0): their bit patterns order like unsigned integers
+      const unsigned sb = scored ? __float_as_uint(score) : 0xffffffffu;
+      const unsigned smin = __reduce_min_sync(0xffffffffu, sb);
+      const unsigned tb_ = (sb == smin && scored) ? (unsigned)(0x7fffffff - pos) : 0xffffffffu;
+      const unsigned tmin = __reduce_min_sync(0xffffffffu, tb_);
+      const unsigned long long k = scored || smin != 0xffffffffu ? (((unsigned long long)smin << 32) | tmin) : ~0ull;
+      const bool is_min = scored && sb == smin && tb_ == tmin;
+      const unsigned s2 = __reduce_min_sync(0xffffffffu, is_min ? 0xffffffffu : sb);
+      const float a1 = smin == 0xffffffffu ? CUDART_INF_F : __uint_as_float(smin);
+      const float a2 = s2 == 0xffffffffu ? CUDART_INF_F : __uint_as_float(s2);
       if (lane == 0) { X.redkey[wg][wq] = k; X.red12[wg][wq][0] = a1; X.red12[wg][wq][1] = a2; }
     }
     tc::named_bar_sync(1 + wg, 256);
@@ -459,42 +476,47 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
         X.cand_min2[tile] = a2;
         X.cand_row[tile] = R;
 #pragma unroll
-        for (int r = 0; r < kDecQ; ++r) X.cand_z[tile][r] = z[r];
-#pragma unroll
-        for (int ch = 0; ch < 16; ++ch)
-          X.cand_phi[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_k + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
+        for (int r = 0; r < QR; ++r) X.cand_z[tile][r] = z[r];
       } else {
 #pragma unroll
         for (int ch = 0; ch < d / 8; ++ch)
           X.cand_v[tile][ch] = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
       }
     }
+    if (__any_sync(0xffffffffu, left_out)) {       // its feature row, read back from tensor memory (this thread's half)
+      uint32_t pr[32];
+      tc::tmem_ld32u(tm_phi + lane_addr + hf * 32, pr);
+      if (left_out) {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&X.cand_phi[tile][0]) + hf * 32;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) dst[i] = pr[i];
+      }
+    }
     // ---- softmax weights of the tile (bf16; the sums use the rounded weights): query rows 4 hf .. 4 hf + 3
     {
       bool moved = false;
-      float alpha[kDecQ];
+      float alpha[QR];
 #pragma unroll
-      for (int r = 0; r < kDecQ; ++r) {
+      for (int r = 0; r < QR; ++r) {
         alpha[r] = tc::fast_exp2(m_run[r] - m_new[r]);
         moved = moved || (m_new[r] != m_run[r]);
         lpart[r] *= alpha[r];
         m_run[r] = m_new[r];
       }
 #pragma unroll
-      for (int rr = 0; rr < 4; ++rr) {
-        const int r = hf * 4 + rr;
-        if (r < kDecQ) {
+      for (int r = 0; r < QR; ++r) {          // static indices keep z, m_new, lpart in registers
+        if ((r / (QR / 2)) == hf) {
           float p = (valid && !left_out) ? tc::fast_exp2(z[r] - m_new[r]) : 0.f;
-          const __nv_bfloat16 pb = __float2bfloat16_rn(p);
-          lpart[r] += __bfloat162float(pb);
-          *reinterpret_cast<T*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = pb;
+          const uint32_t pb = pack_bf16x2(p, 0.f);
+          lpart[r] += bf16lo_f(pb);
+          *reinterpret_cast<unsigned short*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = (unsigned short)pb;
         }
       }
       if (have_o && moved && hf == 0) {          // `moved` is uniform over the row group
         float ov[8];
         tc::tmem_ld8(tm_o + lane_addr, ov);
 #pragma unroll
-        for (int r = 0; r < kDecQ; ++r) ov[r] *= alpha[r];
+        for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
         tc::tmem_st8(tm_o + lane_addr, ov);
       }
     }
@@ -502,9 +524,8 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     tc::fence_before_sync();
     tc::named_bar_sync(1 + wg, 256);
     tc::fence_after_sync();
-    // ---- O^T += V^T Pr^T; the key/phi buffer is free for the next tile of this row group
+    // ---- O^T += V^T Pr^T
     if (lead) {
-      if (tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
         tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(stage + S::st_v + ks * 2048, 16384, 1024),
@@ -526,19 +547,19 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   tc::named_bar_sync(1 + wg, 256);              // the leader has seen the last O^T product complete
   tc::fence_after_sync();
 #pragma unroll
-  for (int r = 0; r < kDecQ; ++r) {
+  for (int r = 0; r < QR; ++r) {
     float ls = warp_sum(lpart[r]);
     if (lane == 0) X.wg_l[wg][warp & 7][r] = ls;
     if (t == r && hf == 0) X.wg_m[wg][r] = m_run[r];
   }
-  float* opart = reinterpret_cast<float*>(stage_p + S::st_v);   // [128][kDecQ]
+  float* opart = reinterpret_cast<float*>(stage_p + S::st_v);   // [128][QR]
   if (hf == 0) {
     float ov[8];
 #pragma unroll
-    for (int r = 0; r < kDecQ; ++r) ov[r] = 0.f;
+    for (int r = 0; r < QR; ++r) ov[r] = 0.f;
     if (have_o) tc::tmem_ld8(tm_o + lane_addr, ov);
 #pragma unroll
-    for (int r = 0; r < kDecQ; ++r) opart[t * kDecQ + r] = ov[r];
+    for (int r = 0; r < QR; ++r) opart[t * QR + r] = ov[r];
   }
   tc::fence_before_sync();
   __syncthreads();
@@ -562,6 +583,22 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
   const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
 
+  // ---- Eq. 13: H += phi_fold v_fold^T, s += phi_fold (fp32 additions performed at the L2, no read-back)
+  if (ok) {
+    float* Hgw = L.H + (size_t)unit * D * d;
+    constexpr int per_row = d / 4;
+#pragma unroll 4
+    for (int i = tid; i < D * per_row; i += kDecThreads) {
+      const int j = i / per_row, c4 = (i % per_row) * 4;
+      const float pj = __bfloat162float(phiL[j]);
+      const uint2 vv = *reinterpret_cast<const uint2*>(vL + c4);
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Hgw + (size_t)i * 4), "f"(pj * bf16lo_f(vv.x)),
+                   "f"(pj * bf16hi_f(vv.x)), "f"(pj * bf16lo_f(vv.y)), "f"(pj * bf16hi_f(vv.y))
+                   : "memory");
+    }
+    if (tid < D) atomicAdd(L.s + (size_t)unit * D + tid, __bfloat162float(phiL[tid]));
+  }
+
   // ---- Eq. 14: thread (query row r, value column cc)
   if (ok) {
     const float* op0 = reinterpret_cast<const float*>(sm + S::stage0 + S::st_v);
@@ -574,7 +611,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       float l0 = 0.f, l1 = 0.f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) { l0 += X.wg_l[0][w][r]; l1 += X.wg_l[1][w][r]; }
-      float num = a0 * op0[cc * kDecQ + r] + a1 * op1[cc * kDecQ + r];
+      float num = a0 * op0[cc * QR + r] + a1 * op1[cc * QR + r];
       float den = a0 * l0 + a1 * l1;
       for (int ti = 0; ti < NT; ++ti) {
         if (ti == lt || X.cand_key[ti] == ~0ull) continue;
@@ -590,24 +627,6 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       den = fmaf(e, X.lden[r] + X.dotL[r], den);
       ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
     }
-  }
-
-  // ---- Eq. 13: H += phi_fold v_fold^T, s += phi_fold
-  if (ok) {
-    float4* Hg = reinterpret_cast<float4*>(L.H + (size_t)unit * D * d);
-    constexpr int per_row = d / 4;
-#pragma unroll 4
-    for (int i = tid; i < D * per_row; i += kDecThreads) {
-      const int j = i / per_row, c4 = (i % per_row) * 4;
-      const float pj = __bfloat162float(phiL[j]);
-      float4 hv = Hg[i];
-      hv.x = fmaf(pj, __bfloat162float(vL[c4]), hv.x);
-      hv.y = fmaf(pj, __bfloat162float(vL[c4 + 1]), hv.y);
-      hv.z = fmaf(pj, __bfloat162float(vL[c4 + 2]), hv.z);
-      hv.w = fmaf(pj, __bfloat162float(vL[c4 + 3]), hv.w);
-      Hg[i] = hv;
-    }
-    if (tid < D) L.s[(size_t)unit * D + tid] += __bfloat162float(phiL[tid]);
   }
 
   // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself)
