@@ -16,6 +16,8 @@
 #include "lola_score_tc.cuh"
 #include "lola_attend_tc.cuh"
 #include "lola_decode_tc.cuh"
+#include "lola_score2_tc.cuh"
+#include "lola_update2_tc.cuh"
 
 using namespace lola;
 
@@ -149,6 +151,7 @@ struct lola_state {
   int64_t launches;
   bool tensor_path = false;            // bf16, F = 64: tcgen05 kernels
   bool fused_decode = false;           // shapes the one-kernel generation step is built for
+  bool have_maps = false;              // TMA descriptors of the sparse cache and the window ring exist
   bool force_chain = false;            // set while lola_decode_step_static runs: kernel chain with work lists
   CUtensorMap tm_gk, tm_gv, tm_wk, tm_wv;
   bool profiling = false;
@@ -194,6 +197,24 @@ template <typename T, int DPL>
 int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   const int U = L.B * L.Hkv;
+  // chunkwise update on TMA-fed tensor-core kernels: every leaving pair already sits in the ring, the
+  // occupied part of the sparse cache is a whole number of 64-slot blocks
+  if (c.mode == UPD_SELECT && st->have_maps && !st->force_chain && c.count_g % 64 == 0 &&
+      c.r_pos0 + c.r <= c.n_seen && c.count_g + c.r <= kUp2MaxE && c.r <= kUp2MaxFold) {
+    const int NT = (c.count_g / 64 + (L.eta + 63) / 64 + 1) / 2;
+    int tpc = (U * NT + 147) / 148;
+    tpc = std::max(2, tpc + (tpc & 1));
+    const uint4* img = (const uint4*)(st->base + st->lay.wt);
+    {
+      LaunchScope scope(st, LOLA_KERNEL_SCORE, s);
+      dim3 grid((NT + tpc - 1) / tpc, U);
+      k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, tpc);
+      if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
+    }
+    LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+    k_update2_tc<DPL><<<U, kUp2Threads, Update2Smem<DPL>::bytes, s>>>(L, c, img);
+    return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+  }
   if (c.mode == UPD_SELECT) {
     const int nE = c.count_g + c.r;
     dim3 grid((nE + kScoreRows - 1) / kScoreRows, U);
@@ -318,25 +339,29 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
         : cudaFuncSetAttribute(k_attend_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttendTcSmem<2>::bytes);
     if (e != cudaSuccess) rc = LOLA_ERR_CUDA;
   }
-  // one-kernel generation step: lambda a whole number of 64-row blocks, the row stream within 16 tiles
-  st->fused_decode = st->tensor_path && cfg->sparse >= 64 && cfg->sparse % 64 == 0 && cfg->window >= 1 &&
-                     L.g <= kDecQ && (cfg->sparse / 64 + (cfg->window + 63) / 64 + 1) / 2 <= kDecMaxTiles;
-  if (rc == LOLA_OK && st->fused_decode) {
+  if (rc == LOLA_OK && st->tensor_path && cfg->sparse >= 1 && cfg->window >= 1) {
     const size_t U = (size_t)cfg->batch * cfg->n_kv_heads;
-    bool ok = make_rows_map(&st->tm_gk, L.gk, U, cfg->sparse, cfg->head_dim, 64) &&
-              make_rows_map(&st->tm_gv, L.gv, U, cfg->sparse, cfg->head_dim, 64) &&
-              make_rows_map(&st->tm_wk, L.wk, U, cfg->window, cfg->head_dim, 64) &&
-              make_rows_map(&st->tm_wv, L.wv, U, cfg->window, cfg->head_dim, 64);
-    cudaError_t e = cudaSuccess, e2 = cudaSuccess;
+    st->have_maps = make_rows_map(&st->tm_gk, L.gk, U, cfg->sparse, cfg->head_dim, 64) &&
+                    make_rows_map(&st->tm_gv, L.gv, U, cfg->sparse, cfg->head_dim, 64) &&
+                    make_rows_map(&st->tm_wk, L.wk, U, cfg->window, cfg->head_dim, 64) &&
+                    make_rows_map(&st->tm_wv, L.wv, U, cfg->window, cfg->head_dim, 64);
+    cudaError_t e[8];
     if (cfg->head_dim == 128) {
-      e = cudaFuncSetAttribute(k_decode_tc<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
-      e2 = cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
+      e[0] = cudaFuncSetAttribute(k_decode_tc<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
+      e[1] = cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
+      e[2] = cudaFuncSetAttribute(k_score2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<4>::bytes);
+      e[3] = cudaFuncSetAttribute(k_update2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<4>::bytes);
     } else {
-      e = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
-      e2 = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+      e[0] = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+      e[1] = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+      e[2] = cudaFuncSetAttribute(k_score2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<2>::bytes);
+      e[3] = cudaFuncSetAttribute(k_update2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<2>::bytes);
     }
-    if (!ok || e != cudaSuccess || e2 != cudaSuccess) st->fused_decode = false;   // the kernel chain serves every shape
+    for (int i = 0; i < 4; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
   }
+  // one-kernel generation step: lambda a whole number of 64-row blocks, the row stream within 16 tiles
+  st->fused_decode = st->have_maps && cfg->sparse >= 64 && cfg->sparse % 64 == 0 && L.g <= kDecQ &&
+                     (cfg->sparse / 64 + (cfg->window + 63) / 64 + 1) / 2 <= kDecMaxTiles;
   if (rc == LOLA_OK && st->tensor_path) {
     cudaStream_t s = (cudaStream_t)stream;
     __nv_bfloat16* img = (__nv_bfloat16*)(st->base + lay.wt);

@@ -1,0 +1,251 @@
+// Eq. 10 for the chunkwise update (bf16 layer, F = 64): the self-recall error of every member of the
+// sparse cache and of every pair leaving the window, against the H, s before the fold.
+//
+// Rows are streamed by TMA in tiles of 128: sparse-cache slots 0..count_g-1 (count_g a multiple of
+// 64), then the window ring slots 0..eta-1.  One CTA takes `tiles_per_cta` consecutive tiles of one
+// unit; its two row groups of 256 threads (two threads per row) work on alternate tiles:
+//     U = K_tile W                        tcgen05.mma  M=128, N=64,   K=d
+//     phi = feature map of U, rounded to bf16, kept in tensor memory (A operand of the next product)
+//     [P | den] = phi [H | s_hi s_lo]      tcgen05.mma  M=128, N=d+16, K=128
+//     score = || P / den - v ||
+// Ring rows whose pair stays in the window are computed and dropped.
+// Every wait on an mbarrier is bounded; a wait that runs out sets bit 16 of the status word.
+#pragma once
+#include <cuda.h>
+
+#include "lola_decode_tc.cuh"
+#include "lola_generic.cuh"
+#include "lola_tc.cuh"
+
+namespace lola {
+
+constexpr int kSc2Threads = 512;
+
+template <int DPL>
+struct Score2Smem {
+  static constexpr int d = DPL * 32;
+  static constexpr int kblk = d / 64;
+  static constexpr uint32_t b1 = 0;                                  // W^T, K-major: [kblk][64][128B]
+  static constexpr uint32_t ht_blk = (d + 16) * 128;
+  static constexpr uint32_t ht = 16384;                              // [2 j blocks][d + 16 rows][128B]
+  static constexpr uint32_t stage0 = ht + 2 * (128 + 16) * 128;
+  static constexpr uint32_t st_k = 0, st_v = 32768;
+  static constexpr uint32_t stage_bytes = 65536;
+  static constexpr uint32_t misc = stage0 + 2 * stage_bytes;
+  static constexpr uint32_t total = misc + 2048;
+  static constexpr uint32_t bytes = total + 1024;
+};
+
+struct Score2Misc {
+  float ssp[2][128];
+  uint64_t bars[8];
+  uint32_t tmem_slot;
+};
+
+template <int DPL>
+__global__ void __launch_bounds__(kSc2Threads, 1)
+k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
+            const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image,
+            int tiles_per_cta) {
+  using S = Score2Smem<DPL>;
+  constexpr int d = DPL * 32;
+  constexpr int kblk = d / 64;
+  constexpr int D = 128;
+  constexpr int HC = d / 2;
+  constexpr float kLog2e = 1.4426950408889634f;
+  typedef __nv_bfloat16 T;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = tc::smem_u32(sm);
+  Score2Misc& X = *reinterpret_cast<Score2Misc*>(sm + S::misc);
+
+  const int unit = blockIdx.y, h = unit % L.Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int wg = tid >> 8, wq = warp & 3, hf = (warp >> 2) & 1;
+  const int t = wq * 32 + lane;
+  const bool lead = (tid & 255) == 0;
+  const int lam = L.lam, eta = L.eta;
+  const int cg = c.count_g;                                // multiple of 64
+  const int nGB = cg / 64, nRB = (eta + 63) / 64, NT = (nGB + nRB + 1) / 2;
+  const int tile0 = blockIdx.x * tiles_per_cta;
+  const int tile1 = min(NT, tile0 + tiles_per_cta);
+  const int cw = min(eta, c.n_seen);                       // pairs in the window before this call
+  const int w0 = c.n_seen - cw;                            // oldest position in the window
+  float* scu = L.score + (size_t)unit * (lam + L.cmax);
+
+  const uint32_t bar_k = sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + (uint32_t)wg * 24u;
+  const uint32_t bar_v = bar_k + 8, bar_mma = bar_k + 16;
+  const uint32_t stage = sbase + S::stage0 + (uint32_t)wg * S::stage_bytes;
+  uint8_t* stage_p = sm + S::stage0 + (size_t)wg * S::stage_bytes;
+  uint32_t pk = 0, pv = 0, pm = 0;
+  bool ok = true;
+
+  if (tid == 0) {
+    for (int i = 0; i < 6; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 8u * i, 1);
+    tc::mbar_init_fence();
+  }
+  if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
+  __syncthreads();
+  if (lead && tile0 + wg < tile1) {
+    decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile0 + wg, nGB, nRB, unit, bar_k);
+    decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile0 + wg, nGB, nRB, unit, bar_v);
+  }
+  // ---- operands: H^T (bf16, K-major) with the two parts of s as rows d, d+1; W^T image
+  {
+    constexpr int HI = d * (D / 8) / kSc2Threads;
+    float hreg[HI][8];
+    const float* Hg = L.H + (size_t)unit * D * d;
+#pragma unroll
+    for (int it = 0; it < HI; ++it) {
+      const int i = tid + it * kSc2Threads;
+      const int cc = i % d, jc = i / d;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) hreg[it][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+    }
+    const uint4* img = wt_image + (size_t)h * kblk * 512;
+    for (int i = tid; i < kblk * 512; i += kSc2Threads)
+      *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
+    if (tid < D) {
+      const float sv = L.s[(size_t)unit * D + tid];
+      const __nv_bfloat16 hi = __float2bfloat16_rn(sv);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(sv - __bfloat162float(hi));
+      const int ch = (tid & 63) >> 3;
+      *reinterpret_cast<T*>(sm + S::ht + (tid >> 6) * S::ht_blk + tc::sw128_off(d, ch) + (tid & 7) * 2) = hi;
+      *reinterpret_cast<T*>(sm + S::ht + (tid >> 6) * S::ht_blk + tc::sw128_off(d + 1, ch) + (tid & 7) * 2) = lo;
+    }
+    for (int i = tid; i < 2 * 14 * 8; i += kSc2Threads) {
+      const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
+      *reinterpret_cast<uint4*>(sm + S::ht + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int it = 0; it < HI; ++it) {
+      const int i = tid + it * kSc2Threads;
+      const int cc = i % d, jc = i / d;
+      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(hreg[it]);
+    }
+  }
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem = X.tmem_slot;
+  const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+  const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // U, then [P | den]
+  const uint32_t tm_phi = tm_a + 192u;
+  const uint32_t idesc1 = tc::make_idesc_bf16(128, 64, false, false);
+  const uint32_t idesc2 = tc::make_idesc_bf16(128, d + 16, false, false);
+
+  if (wg == 1) asm volatile("bar.arrive 3, 512;" ::: "memory");   // row group 0 takes the first turn
+
+  for (int tile = tile0 + wg; tile < tile1; tile += 2) {
+    const int R = tile * 128 + t;
+    const bool is_g = R < cg;
+    const int slot = R - cg;
+    // ring slot -> position it holds; it is scored if that pair leaves the window in this call
+    int e_idx = -1;
+    if (is_g) e_idx = R;
+    else if (slot < eta) {
+      int off = slot - (w0 % eta);
+      if (off < 0) off += eta;
+      const int p = w0 + off;
+      if (off < cw && p < c.r_pos0 + c.r && p >= c.r_pos0) e_idx = lam + (p - c.r_pos0);
+    }
+
+    ok = tc::mbar_wait(bar_k, pk) && ok; pk ^= 1;
+    tc::fence_after_sync();
+    if (lead) {
+#pragma unroll
+      for (int ks = 0; ks < d / 16; ++ks)
+        tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                        tc::make_desc_sw128(sbase + S::b1 + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), idesc1, ks > 0);
+      tc::mma_commit(bar_mma);
+    }
+    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
+    tc::fence_after_sync();
+    if (lead && tile + 2 < tile1) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
+    {
+      tc::named_bar_sync(3 + wg, 512);
+      float e[64];
+      tc::tmem_ld64(tm_a + lane_addr, e);
+      const float sgn = hf ? -kLog2e : kLog2e;
+      if (L.phi_kind == 1) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
+      } else {
+        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
+#pragma unroll
+        for (int i = 0; i < 64; i += 4) {
+          m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn);
+          m2 = fmaxf(m2, e[i + 2] * sgn); m3 = fmaxf(m3, e[i + 3] * sgn);
+        }
+        const float mm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 64; i += 4) {
+          e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
+          e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
+          e[i + 2] = tc::fast_exp2(fmaf(e[i + 2], sgn, -mm)); s2 += e[i + 2];
+          e[i + 3] = tc::fast_exp2(fmaf(e[i + 3], sgn, -mm)); s3 += e[i + 3];
+        }
+        const float inv = 1.0f / ((s0 + s1) + (s2 + s3));
+#pragma unroll
+        for (int i = 0; i < 64; ++i) e[i] *= inv;
+      }
+      uint32_t pk2[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) pk2[i] = pack_bf16x2(e[2 * i], e[2 * i + 1]);
+      tc::tmem_st32u(tm_phi + lane_addr + hf * 32, pk2);
+      if (wg == 0) asm volatile("bar.arrive 4, 512;" ::: "memory"); else asm volatile("bar.arrive 3, 512;" ::: "memory");
+    }
+    tc::fence_before_sync();
+    tc::named_bar_sync(1 + wg, 256);
+    tc::fence_after_sync();
+    if (lead) {
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks)
+        tc::mma_bf16_ts(tm_a, tm_phi + ks * 8,
+                        tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024), idesc2, ks > 0);
+      tc::mma_commit(bar_mma);
+    }
+    ok = tc::mbar_wait(bar_v, pv) && ok; pv ^= 1;
+    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
+    tc::fence_after_sync();
+    {
+      float dn[2];
+      tc::tmem_ld2(tm_a + lane_addr + d, dn);
+      const float den = dn[0] + dn[1];
+      const float inv = den > 0.f ? 1.0f / den : 0.f;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+      for (int c0 = 0; c0 < HC; c0 += 32) {
+        float p[32];
+        tc::tmem_ld32(tm_a + lane_addr + hf * HC + c0, p);
+#pragma unroll
+        for (int q8 = 0; q8 < 4; ++q8) {
+          const int cc = hf * HC + c0 + q8 * 8;
+          uint4 raw = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (cc >> 6) * 16384 + tc::sw128_off(t, (cc & 63) >> 3));
+          float d0 = fmaf(p[q8 * 8 + 0], inv, -bf16lo_f(raw.x)), d1 = fmaf(p[q8 * 8 + 1], inv, -bf16hi_f(raw.x));
+          float d2 = fmaf(p[q8 * 8 + 2], inv, -bf16lo_f(raw.y)), d3 = fmaf(p[q8 * 8 + 3], inv, -bf16hi_f(raw.y));
+          float d4 = fmaf(p[q8 * 8 + 4], inv, -bf16lo_f(raw.z)), d5 = fmaf(p[q8 * 8 + 5], inv, -bf16hi_f(raw.z));
+          float d6 = fmaf(p[q8 * 8 + 6], inv, -bf16lo_f(raw.w)), d7 = fmaf(p[q8 * 8 + 7], inv, -bf16hi_f(raw.w));
+          a0 = fmaf(d0, d0, a0); a1 = fmaf(d1, d1, a1); a2 = fmaf(d2, d2, a2); a3 = fmaf(d3, d3, a3);
+          a0 = fmaf(d4, d4, a0); a1 = fmaf(d5, d5, a1); a2 = fmaf(d6, d6, a2); a3 = fmaf(d7, d7, a3);
+        }
+      }
+      const float ss = (a0 + a1) + (a2 + a3);
+      if (hf == 1) X.ssp[wg][t] = ss;
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      tc::named_bar_sync(1 + wg, 256);          // both halves are done with the value tile and with P
+      tc::fence_after_sync();
+      if (hf == 0 && e_idx >= 0 && ok) scu[e_idx] = sqrtf(ss + X.ssp[wg][t]);
+    }
+    if (lead && tile + 2 < tile1) decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_v);
+  }
+  if (!ok && (tid & 255) == 0) atomicOr(L.status, 16);
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, 512);
+}
+
+}  // namespace lola

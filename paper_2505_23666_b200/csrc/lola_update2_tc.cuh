@@ -1,0 +1,318 @@
+// Eq. 12 and Eq. 13 of the chunkwise update in one kernel (bf16 layer, F = 64), one CTA per unit:
+//   1. exact top-lambda of the eligible set by (score descending, older first): the n_fold = |E| - lambda
+//      lowest keys are found with a 4-pass byte radix select over the score bits; ties on the
+//      threshold score are resolved by position (the younger pair is folded first);
+//   2. ordered compaction into three lists (pairs to fold, freed slots, leaving pairs that stay);
+//   3. the folded pairs are gathered into operand tiles, phi(K_S) is recomputed
+//      (tcgen05.mma K_S W, feature map with one thread pair per row, rounded to bf16) and
+//      [dH | ds] = phi(K_S)^T [V_S | 1]   (tcgen05.mma, M = 128 features, N = d + 16, K = folded pairs)
+//      is added to H, s with vector reductions at the L2;
+//   4. leaving pairs that stay move into the freed slots; the incoming pairs enter the window ring.
+// Every wait on an mbarrier is bounded; a wait that runs out sets bit 32 of the status word.
+#pragma once
+#include <cuda.h>
+
+#include "lola_decode_tc.cuh"
+#include "lola_generic.cuh"
+#include "lola_tc.cuh"
+
+namespace lola {
+
+constexpr int kUp2Threads = 512;
+constexpr int kUp2MaxE = 4096;      // eligible pairs this kernel handles (scores and positions in shared memory)
+constexpr int kUp2MaxFold = 128;    // folded pairs per call (one operand tile)
+
+template <int DPL>
+struct Update2Smem {
+  static constexpr int d = DPL * 32;
+  static constexpr int kblk = d / 64;
+  static constexpr uint32_t b1 = 0;                        // W^T, K-major: [kblk][64][128B]
+  static constexpr uint32_t kt = 16384;                    // K_S tile, K-major [kblk][128][128B]; then phi tile [2][128][128B]
+  static constexpr uint32_t vt = kt + 32768;               // [V_S | 1], MN-major: [kblk + 1 column blocks][128 pairs][128B]
+  static constexpr uint32_t misc = vt + 3 * 16384;
+  static constexpr uint32_t total = misc + 2 * kUp2MaxE * 4 + 8192;
+  static constexpr uint32_t bytes = total + 1024;
+};
+
+struct Update2Misc {
+  unsigned key[kUp2MaxE];           // score bits
+  int pos[kUp2MaxE];                // position; bit 31 set once the pair is chosen for folding
+  unsigned hist[256];
+  int scan[kUp2Threads / 32][3];
+  int fold_e[kUp2MaxFold];          // E indices of the folded pairs, ascending
+  int free_slot[kUp2MaxFold];       // sparse-cache slots of folded members, ascending
+  int mover[kUp2MaxFold];           // leaving-pair indices that stay, ascending
+  unsigned sel_prefix, sel_need, min_keep;
+  int n_equal_fold;
+  uint64_t bars[2];
+  uint32_t tmem_slot;
+};
+static_assert(sizeof(Update2Misc) <= 2 * kUp2MaxE * 4 + 8192, "misc region too small");
+
+template <int DPL>
+__global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image) {
+  using S = Update2Smem<DPL>;
+  constexpr int d = DPL * 32;
+  constexpr int kblk = d / 64;
+  constexpr int D = 128;
+  constexpr int nch = d / 8;
+  constexpr float kLog2e = 1.4426950408889634f;
+  typedef __nv_bfloat16 T;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = tc::smem_u32(sm);
+  Update2Misc& X = *reinterpret_cast<Update2Misc*>(sm + S::misc);
+
+  const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int lam = L.lam, eta = L.eta;
+  const int cg = c.count_g, nE = cg + c.r, nF = nE - lam;          // 1 <= nF <= min(r, kUp2MaxFold)
+  float* scu = L.score + (size_t)unit * (lam + L.cmax);
+  const uint32_t bar = sbase + S::misc + (uint32_t)offsetof(Update2Misc, bars);
+  uint32_t ph = 0;
+  bool ok = true;
+
+  if (tid == 0) { tc::mbar_init(bar, 1); tc::mbar_init_fence(); X.min_keep = 0xffffffffu; X.n_equal_fold = 0; }
+  if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
+  // W^T image and zeroed operand tiles can be staged while the selection runs
+  {
+    const uint4* img = wt_image + (size_t)h * kblk * 512;
+    for (int i = tid; i < kblk * 512; i += kUp2Threads) *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
+    for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
+      *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
+  }
+  for (int e = tid; e < nE; e += kUp2Threads) {
+    if (e < cg) { X.key[e] = __float_as_uint(scu[e]); X.pos[e] = L.gpos[(size_t)unit * lam + e]; }
+    else { X.key[e] = __float_as_uint(scu[lam + (e - cg)]); X.pos[e] = c.r_pos0 + (e - cg); }
+  }
+  // ---- 1. radix select of the nF lowest scores (scores are norms >= 0: bit patterns order like unsigned)
+  unsigned prefix = 0, mask = 0, need = (unsigned)nF;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) X.hist[tid] = 0;
+    __syncthreads();
+    for (int e = tid; e < nE; e += kUp2Threads) {
+      const unsigned k = X.key[e];
+      if ((k & mask) == prefix) atomicAdd(&X.hist[(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // 8 bins per lane, exclusive scan over the 256 bins
+      unsigned cnt[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { cnt[i] = X.hist[lane * 8 + i]; tot += cnt[i]; }
+      unsigned incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      unsigned run = incl - tot;                     // elements in lower bins
+      if (run < need && need <= incl) {              // exactly one lane holds the bin of the need-th lowest
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (run < need && need <= run + cnt[i]) {
+            X.sel_prefix = prefix | ((unsigned)(lane * 8 + i) << shift);
+            X.sel_need = need - run;
+          }
+          run += cnt[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = X.sel_prefix;
+    need = X.sel_need;
+    mask |= 255u << shift;
+  }
+  // prefix = the nF-th lowest score; `need` of the pairs with exactly that score are folded: the youngest
+  const unsigned thr_key = prefix;
+  for (int e = tid; e < nE; e += kUp2Threads) {
+    const unsigned k = X.key[e];
+    bool fold = k < thr_key;
+    if (k == thr_key) {
+      const int pe = X.pos[e] & 0x7fffffff;
+      unsigned younger = 0;
+      for (int j = 0; j < nE; ++j) younger += (X.key[j] == thr_key && (X.pos[j] & 0x7fffffff) > pe) ? 1u : 0u;
+      fold = younger < need;
+    }
+    if (!fold) atomicMin(&X.min_keep, k);
+    // mark (other threads read pos only through the 31-bit mask above)
+    if (fold) atomicOr(reinterpret_cast<unsigned*>(&X.pos[e]), 0x80000000u);
+  }
+  __syncthreads();
+  // ---- 2. ordered compaction: each thread owns a contiguous range of E
+  {
+    const int per = (nE + kUp2Threads - 1) / kUp2Threads;
+    const int e0 = min(nE, tid * per), e1 = min(nE, e0 + per);
+    int nf = 0, ng = 0, nm = 0;                      // folded, folded members of G, leaving pairs that stay
+    for (int e = e0; e < e1; ++e) {
+      const bool fold = X.pos[e] < 0;
+      nf += fold ? 1 : 0;
+      ng += (fold && e < cg) ? 1 : 0;
+      nm += (!fold && e >= cg) ? 1 : 0;
+    }
+    int inf = nf, ing = ng, inm = nm;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int a = __shfl_up_sync(0xffffffffu, inf, o), bq = __shfl_up_sync(0xffffffffu, ing, o), cq = __shfl_up_sync(0xffffffffu, inm, o);
+      if (lane >= o) { inf += a; ing += bq; inm += cq; }
+    }
+    if (lane == 31) { X.scan[warp][0] = inf; X.scan[warp][1] = ing; X.scan[warp][2] = inm; }
+    __syncthreads();
+    int bf = 0, bg = 0, bm = 0;
+    for (int w = 0; w < warp; ++w) { bf += X.scan[w][0]; bg += X.scan[w][1]; bm += X.scan[w][2]; }
+    int of = bf + inf - nf, og = bg + ing - ng, om = bm + inm - nm;
+    for (int e = e0; e < e1; ++e) {
+      const bool fold = X.pos[e] < 0;
+      if (fold) {
+        if (of < kUp2MaxFold) X.fold_e[of] = e;
+        ++of;
+        if (e < cg) { if (og < kUp2MaxFold) X.free_slot[og] = e; ++og; }
+      } else if (e >= cg) {
+        if (om < kUp2MaxFold) X.mover[om] = e - cg;
+        ++om;
+      }
+    }
+  }
+  __syncthreads();
+  int nGL = 0, nMove = 0;
+  for (int w = 0; w < kUp2Threads / 32; ++w) { nGL += X.scan[w][1]; nMove += X.scan[w][2]; }
+
+  // ---- 3. gather the folded pairs into the operand tiles (rows >= nF stay zero)
+  for (int i = tid; i < nF * nch * 2; i += kUp2Threads) {
+    const int row = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+    const int e = X.fold_e[row];
+    const T *kp, *vp;
+    locate_eligible<T>(L, c, unit, b, h, e, kp, vp);
+    const uint4 val = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
+    *reinterpret_cast<uint4*>(sm + (isv ? S::vt : S::kt) + (ch >> 3) * 16384 + tc::sw128_off(row, ch & 7)) = val;
+  }
+  if (tid < nF)                                                      // the column of ones (block kblk, column 0)
+    *reinterpret_cast<T*>(sm + S::vt + kblk * 16384 + tc::sw128_off(tid, 0)) = __float2bfloat16_rn(1.0f);
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem = X.tmem_slot;
+  const uint32_t tm_u = tmem, tm_d = tmem + 64;
+  const int wq = warp & 3, hf = (warp >> 2) & 1;
+  const int t = wq * 32 + lane;
+  const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+  if (tid == 0) {
+#pragma unroll
+    for (int ks = 0; ks < d / 16; ++ks)
+      tc::mma_bf16_ss(tm_u, tc::make_desc_sw128(sbase + S::kt + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                      tc::make_desc_sw128(sbase + S::b1 + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024),
+                      tc::make_idesc_bf16(128, 64, false, false), ks > 0);
+    tc::mma_commit(bar);
+  }
+  ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1;
+  tc::fence_after_sync();
+  if (tid < 256) {                                                   // one thread pair per row: half of the feature map each
+    float e[64];
+    tc::tmem_ld64(tm_u + lane_addr, e);
+    const float sgn = hf ? -kLog2e : kLog2e;
+    if (L.phi_kind == 1) {
+#pragma unroll
+      for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
+    } else {
+      float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
+#pragma unroll
+      for (int i = 0; i < 64; i += 4) {
+        m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn);
+        m2 = fmaxf(m2, e[i + 2] * sgn); m3 = fmaxf(m3, e[i + 3] * sgn);
+      }
+      const float mm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+      for (int i = 0; i < 64; i += 4) {
+        e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
+        e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
+        e[i + 2] = tc::fast_exp2(fmaf(e[i + 2], sgn, -mm)); s2 += e[i + 2];
+        e[i + 3] = tc::fast_exp2(fmaf(e[i + 3], sgn, -mm)); s3 += e[i + 3];
+      }
+      const float inv = 1.0f / ((s0 + s1) + (s2 + s3));
+#pragma unroll
+      for (int i = 0; i < 64; ++i) e[i] *= inv;
+    }
+    // phi tile over the key tile (consumed): row = folded pair, 64 features per 128-byte row and block
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+      uint4 o;
+      o.x = pack_bf16x2(e[ch * 8], e[ch * 8 + 1]);
+      o.y = pack_bf16x2(e[ch * 8 + 2], e[ch * 8 + 3]);
+      o.z = pack_bf16x2(e[ch * 8 + 4], e[ch * 8 + 5]);
+      o.w = pack_bf16x2(e[ch * 8 + 6], e[ch * 8 + 7]);
+      *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t, ch)) = o;
+    }
+  }
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  if (tid == 0) {
+    // [dH | ds] = phi^T [V | 1]: A = phi tile read MN-major (M = feature), B = value tile MN-major
+    const int ksteps = (nF + 15) / 16;
+    for (int ks = 0; ks < ksteps; ++ks)
+      tc::mma_bf16_ss(tm_d, tc::make_desc_sw128(sbase + S::kt + ks * 2048, 16384, 1024),
+                      tc::make_desc_sw128(sbase + S::vt + ks * 2048, 16384, 1024),
+                      tc::make_idesc_bf16(128, d + 16, true, true), ks > 0);
+    tc::mma_commit(bar);
+  }
+  ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1;
+  tc::fence_after_sync();
+  if (tid < 256 && ok) {                                             // row j = t, columns [hf * d/2, +d/2)
+    constexpr int HC = d / 2;
+    float* Hrow = L.H + ((size_t)unit * D + t) * d + hf * HC;
+#pragma unroll
+    for (int c0 = 0; c0 < HC; c0 += 32) {
+      float p[32];
+      tc::tmem_ld32(tm_d + lane_addr + hf * HC + c0, p);
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Hrow + c0 + q * 4), "f"(p[q * 4]), "f"(p[q * 4 + 1]),
+                     "f"(p[q * 4 + 2]), "f"(p[q * 4 + 3])
+                     : "memory");
+    }
+    if (hf == 0) {
+      float ds[2];
+      tc::tmem_ld2(tm_d + lane_addr + d, ds);
+      atomicAdd(L.s + (size_t)unit * D + t, ds[0]);
+    }
+  }
+  // ---- 4. leaving pairs that stay: into the freed slots, then into the slots beyond count_g
+  for (int i = tid; i < nMove * nch * 2; i += kUp2Threads) {
+    const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+    const int src = X.mover[w];
+    const int dst = w < nGL ? X.free_slot[w] : cg + (w - nGL);
+    const T *kp, *vp;
+    locate_leaving<T>(L, c, unit, b, h, c.r_pos0 + src, kp, vp);
+    T* dp = (isv ? (T*)L.gv : (T*)L.gk) + ((size_t)unit * lam + dst) * d;
+    *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
+    if (rem == 0) {
+      L.gpos[(size_t)unit * lam + dst] = c.r_pos0 + src;
+      scu[dst] = scu[lam + src];
+    }
+  }
+  if (tid == 0 && ok) {
+    L.thr[(size_t)unit * 2 + 0] = __uint_as_float(X.min_keep);
+    L.thr[(size_t)unit * 2 + 1] = __uint_as_float(thr_key);
+  }
+  __syncthreads();                                                   // ring rows are read above before they are replaced
+  if (eta > 0) {
+    const int first = max(0, c.n - eta);
+    for (int i = tid; i < (c.n - first) * nch * 2; i += kUp2Threads) {
+      const int ci = first + i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+      const int p = c.n_seen + ci;
+      const T* sp = (isv ? (const T*)c.v : (const T*)c.k) + (((size_t)b * c.n + ci) * L.Hkv + h) * d;
+      T* dp = (isv ? (T*)L.wv : (T*)L.wk) + ((size_t)unit * eta + (p % eta)) * d;
+      *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>(sp + ch * 8);
+    }
+  }
+  if (!ok && tid == 0) atomicOr(L.status, 32);
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, 256);
+}
+
+}  // namespace lola
