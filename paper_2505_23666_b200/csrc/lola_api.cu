@@ -18,6 +18,7 @@
 #include "lola_decode_tc.cuh"
 #include "lola_score2_tc.cuh"
 #include "lola_update2_tc.cuh"
+#include "lola_attend2_tc.cuh"
 
 using namespace lola;
 
@@ -138,6 +139,20 @@ bool make_rows_map(CUtensorMap* tm, void* base, size_t units, size_t rows, size_
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 tensor [B][n][heads][d] of one call viewed as rank 4 (d, head, token, batch row); boxes of 64
+// columns x 1 head x 64 tokens, 128-byte swizzle.  Tokens beyond n read as zeros.
+bool make_tokens_map(CUtensorMap* tm, const void* base, size_t B, size_t n, size_t heads, size_t d) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {d, heads, n, B};
+  cuuint64_t strides[3] = {d * 2, heads * d * 2, n * heads * d * 2};
+  cuuint32_t box[4] = {64, 1, 64, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 struct ProfRecord { int kind; cudaEvent_t a, b; };
@@ -183,6 +198,18 @@ template <typename T, int DPL>
 int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   dim3 grid((L.g * c.nq + kAttRows - 1) / kAttRows, L.B * L.Hkv);
+  if (st->have_maps && !st->force_chain && c.att_chunk == c.nq && c.nq <= 64 && c.n == c.nq) {
+    // prefill chunk: TMA-fed, warp-specialised kernel; the call's q, k, v get their own descriptors
+    CUtensorMap tq, tk, tv;
+    if (make_tokens_map(&tq, c.q, L.B, c.nq, L.Hq, L.d) && make_tokens_map(&tk, c.k, L.B, c.n, L.Hkv, L.d) &&
+        make_tokens_map(&tv, c.v, L.B, c.n, L.Hkv, L.d)) {
+      LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
+      dim3 grid2(((L.g + 1) / 2 + 1) / 2, L.B * L.Hkv);
+      k_attend2_tc<DPL><<<grid2, kAt2Threads, Attend2Smem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, tq, tk,
+                                                                            tv, (const uint4*)(st->base + st->lay.wt));
+      return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+    }
+  }
   LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
   if (st->tensor_path && L.g * c.nq >= 64) {
     dim3 tgrid((L.g * c.nq + kAtM - 1) / kAtM, L.B * L.Hkv);
@@ -351,13 +378,15 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       e[1] = cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
       e[2] = cudaFuncSetAttribute(k_score2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<4>::bytes);
       e[3] = cudaFuncSetAttribute(k_update2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<4>::bytes);
+      e[4] = cudaFuncSetAttribute(k_attend2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<4>::bytes);
     } else {
       e[0] = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[1] = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[2] = cudaFuncSetAttribute(k_score2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<2>::bytes);
       e[3] = cudaFuncSetAttribute(k_update2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<2>::bytes);
+      e[4] = cudaFuncSetAttribute(k_attend2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<2>::bytes);
     }
-    for (int i = 0; i < 4; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
+    for (int i = 0; i < 5; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
   }
   // one-kernel generation step: lambda a whole number of 64-row blocks, the row stream within 16 tiles
   st->fused_decode = st->have_maps && cfg->sparse >= 64 && cfg->sparse % 64 == 0 && L.g <= kDecQ &&

@@ -1,0 +1,428 @@
+// Eq. 14 for a prefill chunk (bf16 layer, F = 64, at most 64 tokens per call): softmax attention of
+// the chunk's queries over the sparse cache, the resident window and the chunk itself (causal), with
+// the linear term phi(q)^T H and its normaliser phi(q)^T s in the same denominator.
+//
+// One CTA serves up to two query tiles of one unit.  A query tile is 128 rows = two query heads x
+// 64 token slots.  Keys and values stream through two shared-memory stages in tiles of 128 rows
+// (64-row blocks of sparse-cache slots, ring slots, then the incoming chunk), loaded once for both
+// query tiles by TMA.  Warp roles:
+//   warps 0-3 / 4-7  softmax of query tile 0 / 1, one thread per row: S from tensor memory, masked
+//                    maximum (the stabiliser only moves when it must grow by more than 2^8), weights
+//                    exp(z - m) rounded to bf16 and written back over S as the A operand of PV
+//   warp 8           issues every tcgen05.mma:  S_w = Q_w K^T,  O_w += P_w V  (P_w in tensor memory)
+//   warp 9           TMA producer
+// After the last tile the feature map of the queries is computed (U_w = Q_w W on the tensor cores, one
+// thread per row), scaled by exp(-m) and fed as a tensor-memory A operand into O_w += phi H and into
+// phi [s_hi s_lo], so the linear term lands in the same accumulator and denominator.
+// Every wait on an mbarrier is bounded; a wait that runs out sets bit 64 of the status word and makes
+// the other waits of the CTA return at once.
+#pragma once
+#include <cuda.h>
+
+#include "lola_decode_tc.cuh"
+#include "lola_generic.cuh"
+#include "lola_tc.cuh"
+
+namespace lola {
+
+constexpr int kAt2Threads = 320;
+
+template <int DPL>
+struct Attend2Smem {
+  static constexpr int d = DPL * 32;
+  static constexpr int kblk = d / 64;
+  static constexpr uint32_t q = 0;                                   // 2 x [kblk][128][128B]
+  static constexpr uint32_t stage0 = 65536;                          // 2 x (K 32 KB + V 32 KB)
+  static constexpr uint32_t st_k = 0, st_v = 32768, stage_bytes = 65536;
+  static constexpr uint32_t ht_blk = (d + 16) * 128;
+  static constexpr uint32_t misc = stage0 + 2 * stage_bytes;
+  static constexpr uint32_t total = misc + 1024;
+  static constexpr uint32_t bytes = total + 1024;
+};
+
+struct Attend2Misc {
+  uint64_t bars[24];
+  uint32_t tmem_slot;
+  int abort_word;
+};
+// barrier indices
+enum { A2_QFULL = 0, A2_KFULL = 1, A2_VFULL = 3, A2_KEMPTY = 5, A2_VEMPTY = 7, A2_SFULL = 9, A2_PREADY = 11, A2_ODONE = 13, A2_WFULL = 15 };
+
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"((uint64_t)(uintptr_t)src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+template <int DPL>
+__global__ void __launch_bounds__(kAt2Threads, 1)
+k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
+             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
+             const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_ck,
+             const __grid_constant__ CUtensorMap tm_cv, const uint4* wt_image) {
+  using S = Attend2Smem<DPL>;
+  constexpr int d = DPL * 32;
+  constexpr int kblk = d / 64;
+  constexpr int D = 128;
+  constexpr float kLog2e = 1.4426950408889634f;
+  constexpr float kGrow = 8.0f;                       // the stabiliser moves only when it must grow by more than 2^8
+  typedef __nv_bfloat16 T;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = tc::smem_u32(sm);
+  Attend2Misc& X = *reinterpret_cast<Attend2Misc*>(sm + S::misc);
+  const uint32_t bar0 = sbase + S::misc + (uint32_t)offsetof(Attend2Misc, bars);
+  auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  volatile int* abortw = &X.abort_word;
+  auto WAIT = [&](int i, uint32_t parity) { return tc::mbar_wait(BAR(i), parity, abortw); };
+
+  if (*reinterpret_cast<volatile int*>(L.status) != 0) return;     // an earlier kernel failed: do nothing
+
+  const int unit = blockIdx.y, b = unit / L.Hkv, h = unit % L.Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = L.g, n = c.nq;
+  const int nqt = (g + 1) / 2;                        // query tiles of the unit
+  const int qt0 = blockIdx.x * 2;
+  const int nw = min(2, nqt - qt0);                   // query tiles of this CTA
+  const int att_g = c.att_g, cw = c.att_wn;
+  const int nGB = (att_g + 63) / 64, nRB = (cw + 63) / 64, NB = nGB + nRB + 1, NT = (NB + 1) / 2;
+  const float sl2 = L.scale * kLog2e;
+  bool ok = true;
+
+  if (tid == 0) {
+    X.abort_word = 0;
+    for (int i = 0; i < 17; ++i) tc::mbar_init(BAR(i), (i == A2_PREADY || i == A2_PREADY + 1) ? 128u : 1u);
+    tc::mbar_init_fence();
+  }
+  if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem = X.tmem_slot;
+
+  // block `blk` of the key stream -> TMA source
+  auto issue_block = [&](uint32_t dst, int blk, bool is_v, uint32_t bar) {
+#pragma unroll
+    for (int cb = 0; cb < kblk; ++cb) {
+      const uint32_t dd = dst + (uint32_t)cb * 16384u;
+      if (blk < nGB) tc::tma_load_3d(dd, is_v ? &tm_gv : &tm_gk, cb * 64, blk * 64, unit, bar);
+      else if (blk < nGB + nRB) tc::tma_load_3d(dd, is_v ? &tm_wv : &tm_wk, cb * 64, (blk - nGB) * 64, unit, bar);
+      else if (blk == nGB + nRB) tc::tma_load_4d(dd, is_v ? &tm_cv : &tm_ck, cb * 64, h, 0, b, bar);
+      else tc::tma_load_4d(dd, is_v ? &tm_cv : &tm_ck, cb * 64, h, 64, b, bar);   // beyond the chunk: zeros
+    }
+  };
+
+  if (warp == 9) {
+    // =============================== TMA producer ===============================
+    if (lane == 0) {
+      // queries: tile w, head slot hs -> rows hs * 64 .. hs * 64 + 63
+      tc::mbar_expect_tx(BAR(A2_QFULL), (uint32_t)nw * kblk * 16384u);
+      for (int w = 0; w < nw; ++w)
+        for (int hs = 0; hs < 2; ++hs) {
+          const int hl = (qt0 + w) * 2 + hs;
+          const int head = hl < g ? h * g + hl : L.Hq;          // a head index outside the tensor reads as zeros
+#pragma unroll
+          for (int cb = 0; cb < kblk; ++cb)
+            tc::tma_load_4d(sbase + S::q + (uint32_t)w * 32768u + (uint32_t)cb * 16384u + (uint32_t)hs * 8192u, &tm_q, cb * 64, head,
+                            0, b, BAR(A2_QFULL));
+        }
+      for (int kt = 0; kt < NT; ++kt) {
+        const int st = kt & 1;
+        const uint32_t stage = sbase + S::stage0 + (uint32_t)st * S::stage_bytes;
+        if (kt >= 2) ok = WAIT(A2_KEMPTY + st, ((kt >> 1) - 1) & 1) && ok;
+        tc::mbar_expect_tx(BAR(A2_KFULL + st), (uint32_t)kblk * 16384u);
+        issue_block(stage + S::st_k, 2 * kt, false, BAR(A2_KFULL + st));
+        issue_block(stage + S::st_k + 8192u, 2 * kt + 1, false, BAR(A2_KFULL + st));
+        if (kt >= 2) ok = WAIT(A2_VEMPTY + st, ((kt >> 1) - 1) & 1) && ok;
+        tc::mbar_expect_tx(BAR(A2_VFULL + st), (uint32_t)kblk * 16384u);
+        issue_block(stage + S::st_v, 2 * kt, true, BAR(A2_VFULL + st));
+        issue_block(stage + S::st_v + 8192u, 2 * kt + 1, true, BAR(A2_VFULL + st));
+      }
+      // W^T image into the key buffer of the stage the last tile does not use
+      {
+        const int so = NT & 1;                                    // stage of tile NT - 2 (or the unused one)
+        const int uses = (NT - so + 1) / 2;                       // tiles that went through stage `so`
+        if (uses >= 1) ok = WAIT(A2_KEMPTY + so, (uses - 1) & 1) && ok;
+        tc::mbar_expect_tx(BAR(A2_WFULL), (uint32_t)kblk * 8192u);
+        bulk_copy_g2s(sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k, wt_image + (size_t)h * kblk * 512, kblk * 8192u,
+                      BAR(A2_WFULL));
+      }
+      if (!ok) atomicOr(L.status, 64);
+    }
+  } else if (warp == 8) {
+    // =============================== MMA issuer ===============================
+    if (lane == 0) {
+      const uint32_t idesc_s = tc::make_idesc_bf16(128, 128, false, false);
+      const uint32_t idesc_pv = tc::make_idesc_bf16(128, d, false, true);
+      auto issue_s = [&](int w, int kt) {
+        const uint32_t stage = sbase + S::stage0 + (uint32_t)(kt & 1) * S::stage_bytes;
+#pragma unroll
+        for (int ks = 0; ks < d / 16; ++ks)
+          tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
+                          tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                          tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
+        tc::mma_commit(BAR(A2_SFULL + w));
+      };
+      auto issue_pv = [&](int w, int kt) {
+        const uint32_t stage = sbase + S::stage0 + (uint32_t)(kt & 1) * S::stage_bytes;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + ks * 8,
+                          tc::make_desc_sw128(stage + S::st_v + ks * 2048, 16384, 1024), idesc_pv, (kt > 0 || ks > 0) ? 1u : 0u);
+        tc::mma_commit(BAR(A2_ODONE + w));
+      };
+      ok = WAIT(A2_QFULL, 0) && ok;
+      ok = WAIT(A2_KFULL + 0, 0) && ok;
+      tc::fence_after_sync();
+      for (int w = 0; w < nw; ++w) issue_s(w, 0);
+      tc::mma_commit(BAR(A2_KEMPTY + 0));
+      for (int kt = 0; kt < NT; ++kt) {
+        const int st = kt & 1;
+        ok = WAIT(A2_VFULL + st, (kt >> 1) & 1) && ok;
+        if (kt + 1 < NT) ok = WAIT(A2_KFULL + (st ^ 1), ((kt + 1) >> 1) & 1) && ok;
+        for (int w = 0; w < nw; ++w) {
+          ok = WAIT(A2_PREADY + w, kt & 1) && ok;
+          tc::fence_after_sync();
+          issue_pv(w, kt);
+          if (kt + 1 < NT) issue_s(w, kt + 1);
+        }
+        tc::mma_commit(BAR(A2_VEMPTY + st));
+        if (kt + 1 < NT) tc::mma_commit(BAR(A2_KEMPTY + (st ^ 1)));
+      }
+      // ---- linear term
+      const int sl = (NT - 1) & 1, so = NT & 1;
+      const uint32_t wt = sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k;
+      const uint32_t ht = sbase + S::stage0 + (uint32_t)sl * S::stage_bytes;
+      ok = WAIT(A2_WFULL, 0) && ok;
+      for (int w = 0; w < nw; ++w) {
+        ok = WAIT(A2_PREADY + w, NT & 1) && ok;                         // H^T staged, S_w free
+        tc::fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < d / 16; ++ks)
+          tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
+                          tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                          tc::make_desc_sw128(wt + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024),
+                          tc::make_idesc_bf16(128, 64, false, false), ks > 0);
+        tc::mma_commit(BAR(A2_SFULL + w));
+      }
+      for (int w = 0; w < nw; ++w) {
+        ok = WAIT(A2_PREADY + w, (NT + 1) & 1) && ok;                   // scaled phi(Q_w) in tensor memory
+        tc::fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint64_t bd = tc::make_desc_sw128(ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024);
+          const uint64_t bs = tc::make_desc_sw128(ht + (ks >> 2) * S::ht_blk + d * 128 + (ks & 3) * 32, 16, 1024);
+          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + 64u + ks * 8, bd,
+                          tc::make_idesc_bf16(128, d, false, false), 1u);
+          tc::mma_bf16_ts(tmem + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + 64u + ks * 8, bs,
+                          tc::make_idesc_bf16(128, 16, false, false), ks > 0);
+        }
+        tc::mma_commit(BAR(A2_ODONE + w));
+      }
+      if (!ok) atomicOr(L.status, 64);
+    }
+  } else if (warp < 4 * nw) {
+    // =============================== softmax, one thread per query row ===============================
+    const int w = warp >> 2, wq = warp & 3;
+    const int t = wq * 32 + lane;                      // row of the query tile = tensor-memory lane
+    const int hl = (qt0 + w) * 2 + (t >> 6), tok = t & 63;
+    const bool row_ok = hl < g && tok < n;
+    const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+    const uint32_t tm_s = tmem + (uint32_t)w * 128u + lane_addr;
+    const uint32_t tm_o = tmem + 256u + (uint32_t)w * 128u + lane_addr;
+    const int nthr = nw * 128;
+    // H (fp32) for the linear term: with both query tiles active the 256 threads issue the loads now
+    // and convert / store them after the last tile; a lone query tile loads them at the end
+    constexpr int HI = d * (D / 8) / 256;
+    float hreg[HI][8];
+    const float* Hg = L.H + (size_t)unit * D * d;
+    if (nw == 2) {
+#pragma unroll
+      for (int it = 0; it < HI; ++it) {
+        const int i = tid + it * 256;
+        const int cc = i % d, jc = i / d;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) hreg[it][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+      }
+    }
+    float m_used = 0.f, l = 0.f;                       // log2 units; m >= 0 is the stabiliser max(0, max z)
+    for (int kt = 0; kt < NT; ++kt) {
+      // valid leading columns of each 64-key block of this tile, for this row
+      int lim[2];
+#pragma unroll
+      for (int hb = 0; hb < 2; ++hb) {
+        const int blk = 2 * kt + hb;
+        int v;
+        if (blk < nGB) v = att_g - blk * 64;
+        else if (blk < nGB + nRB) v = cw - (blk - nGB) * 64;
+        else if (blk == nGB + nRB) v = min(n, tok + 1);
+        else v = 0;
+        lim[hb] = max(0, min(64, v));
+      }
+      ok = WAIT(A2_SFULL + w, kt & 1) && ok;
+      tc::fence_after_sync();
+      float mx = -CUDART_INF_F;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        float sv[32];
+        tc::tmem_ld32(tm_s + c0, sv);
+        const int lm = lim[c0 >> 6] - (c0 & 63);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, j < lm ? sv[j] : -CUDART_INF_F);
+      }
+      const float m_tile = mx * sl2;
+      const bool grow = m_tile > m_used + kGrow;
+      if (__any_sync(0xffffffffu, grow)) {             // rare: rescale what this warp's rows have accumulated
+        const float m_new = grow ? m_tile : m_used;
+        const float alpha = tc::fast_exp2(m_used - m_new);
+        l *= alpha;
+        m_used = m_new;
+        if (kt > 0) {                                  // tensor-memory accesses are warp-wide: every lane takes part
+          ok = WAIT(A2_ODONE + w, (kt - 1) & 1) && ok;
+          tc::fence_after_sync();
+#pragma unroll
+          for (int c0 = 0; c0 < d; c0 += 8) {
+            float ov[8];
+            tc::tmem_ld8(tm_o + c0, ov);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ov[j] *= alpha;
+            tc::tmem_st8(tm_o + c0, ov);
+          }
+        }
+      }
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        float sv[32];
+        tc::tmem_ld32(tm_s + c0, sv);
+        const int lm = lim[c0 >> 6] - (c0 & 63);
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = j < lm ? tc::fast_exp2(fmaf(sv[j], sl2, -m_used)) : 0.f;
+          const float p1 = j + 1 < lm ? tc::fast_exp2(fmaf(sv[j + 1], sl2, -m_used)) : 0.f;
+          const uint32_t pp = pack_bf16x2(p0, p1);
+          l += bf16lo_f(pp) + bf16hi_f(pp);            // the sum uses the weights the product uses
+          pk[j >> 1] = pp;
+        }
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n" ::"r"(
+                tm_s + (c0 >> 1)),
+            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]), "r"(pk[8]), "r"(pk[9]),
+            "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
+            : "memory");
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      tc::fence_before_sync();
+      mbar_arrive(BAR(A2_PREADY + w));
+    }
+    // ---- linear term: wait for the last PV of this tile, stage H^T over the last tile's stage
+    ok = WAIT(A2_ODONE + w, (NT - 1) & 1) && ok;
+    tc::fence_after_sync();
+    tc::named_bar_sync(1, nthr);                       // both query tiles are done with the last stage
+    {
+      const int sl = (NT - 1) & 1;
+      uint8_t* htp = sm + S::stage0 + (size_t)sl * S::stage_bytes;
+      if (nw == 2) {
+#pragma unroll
+        for (int it = 0; it < HI; ++it) {
+          const int i = tid + it * 256;
+          const int cc = i % d, jc = i / d;
+          *reinterpret_cast<uint4*>(htp + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(hreg[it]);
+        }
+      } else {
+        for (int i = tid; i < d * (D / 8); i += 128) {
+          const int cc = i % d, jc = i / d;
+          float f8[8];
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) f8[jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+          *reinterpret_cast<uint4*>(htp + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
+        }
+      }
+      if (tid < D) {
+        const float sv = L.s[(size_t)unit * D + tid];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(sv);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(sv - __bfloat162float(hi));
+        const int ch = (tid & 63) >> 3;
+        *reinterpret_cast<T*>(htp + (tid >> 6) * S::ht_blk + tc::sw128_off(d, ch) + (tid & 7) * 2) = hi;
+        *reinterpret_cast<T*>(htp + (tid >> 6) * S::ht_blk + tc::sw128_off(d + 1, ch) + (tid & 7) * 2) = lo;
+      }
+      for (int i = tid; i < 2 * 14 * 8; i += nthr) {
+        const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
+        *reinterpret_cast<uint4*>(htp + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    tc::named_bar_sync(1, nthr);
+    mbar_arrive(BAR(A2_PREADY + w));                   // phase NT: operands staged, S_w may be overwritten
+    ok = WAIT(A2_SFULL + w, NT & 1) && ok;
+    tc::fence_after_sync();
+    {
+      // phi(q) of this row, scaled by exp(-m): bf16 pairs into columns 64..127 of S_w (A operand)
+      float u[64];
+      tc::tmem_ld64(tm_s, u);
+      const float em = tc::fast_exp2(-m_used);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float e[64];
+        const float sgn = half ? -kLog2e : kLog2e;
+        float scale;
+        if (L.phi_kind == 1) {
+#pragma unroll
+          for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(u[i] * sgn);
+          scale = em;
+        } else {
+          float mm = -CUDART_INF_F;
+#pragma unroll
+          for (int i = 0; i < 64; ++i) mm = fmaxf(mm, u[i] * sgn);
+          float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+          for (int i = 0; i < 64; i += 2) {
+            e[i] = tc::fast_exp2(fmaf(u[i], sgn, -mm)); s0 += e[i];
+            e[i + 1] = tc::fast_exp2(fmaf(u[i + 1], sgn, -mm)); s1 += e[i + 1];
+          }
+          scale = em / (s0 + s1);
+        }
+        uint32_t pk2[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) pk2[i] = pack_bf16x2(e[2 * i] * scale, e[2 * i + 1] * scale);
+        tc::tmem_st32u(tm_s + 64 + half * 32, pk2);
+      }
+    }
+    tc::fence_before_sync();
+    mbar_arrive(BAR(A2_PREADY + w));                   // phase NT + 1
+    ok = WAIT(A2_ODONE + w, NT & 1) && ok;
+    tc::fence_after_sync();
+    {
+      float dn[2];
+      tc::tmem_ld2(tm_s, dn);
+      const float inv = 1.0f / (l + dn[0] + dn[1]);
+      T* op = (T*)c.out + (((size_t)b * n + tok) * L.Hq + h * g + hl) * d;
+#pragma unroll
+      for (int c0 = 0; c0 < d; c0 += 32) {
+        float ov[32];
+        tc::tmem_ld32(tm_o + c0, ov);
+        if (row_ok && ok) {
+#pragma unroll
+          for (int q8 = 0; q8 < 4; ++q8) {
+            uint4 o;
+            o.x = pack_bf16x2(ov[q8 * 8 + 0] * inv, ov[q8 * 8 + 1] * inv);
+            o.y = pack_bf16x2(ov[q8 * 8 + 2] * inv, ov[q8 * 8 + 3] * inv);
+            o.z = pack_bf16x2(ov[q8 * 8 + 4] * inv, ov[q8 * 8 + 5] * inv);
+            o.w = pack_bf16x2(ov[q8 * 8 + 6] * inv, ov[q8 * 8 + 7] * inv);
+            *reinterpret_cast<uint4*>(op + c0 + q8 * 8) = o;
+          }
+        }
+      }
+    }
+    if (!ok && t == 0) atomicOr(L.status, 64);
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, 512);
+}
+
+}  // namespace lola

@@ -141,10 +141,19 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
-// Waits for the phase with the given parity to complete.  Gives up after a bounded number of polls
-// (about a second) and returns false; the caller records the failure and carries on to its cleanup.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < (1u << 24); ++it) {
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Waits for the phase with the given parity to complete.  Gives up after about a quarter of a second
+// and returns false; the caller records the failure and carries on to its cleanup.  With an abort
+// word (shared memory) the first wait that gives up raises it and every other wait of the CTA that
+// polls it returns false at once, so one lost signal cannot add up to many timeouts.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word = nullptr) {
+  unsigned long long deadline = 0;
+  for (uint32_t it = 0;; ++it) {
     uint32_t done;
     asm volatile(
         "{\n\t"
@@ -157,8 +166,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     if (done) return true;
     if (it > 64) __nanosleep(64);
+    if ((it & 255u) == 255u) {
+      if (abort_word && *abort_word) return false;
+      const unsigned long long now = global_ns();
+      if (deadline == 0) deadline = now + 250000000ull;
+      else if (now > deadline) {
+        if (abort_word) *abort_word = 1;
+        return false;
+      }
+    }
   }
-  return false;
 }
 
 // ---- TMA (bulk tensor copies global -> shared, completion on an mbarrier) ------------------------
