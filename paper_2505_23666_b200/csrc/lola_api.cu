@@ -28,7 +28,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct StateLayout {
-  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, wt, total;
+  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, himg, wt, total;
 };
 
 bool config_ok(const lola_config* c) {
@@ -67,7 +67,9 @@ StateLayout make_layout(const lola_config& c) {
   l.move_dst = take(U * cm * 4);
   l.counts = take(U * 4 * 4);
   l.thr = take(U * 2 * 4);
-  // W^T of every KV head in tensor-core operand layout (bf16 layers with F = 64 only)
+  // H of every unit as a bf16 tensor-core operand image, then W^T of every KV head in operand layout
+  // (bf16 layers with F = 64 only)
+  l.himg = take(c.dtype == LOLA_BF16 && c.feat_half == 64 ? U * 2 * d * 64 * 2 : 0);
   l.wt = take(c.dtype == LOLA_BF16 && c.feat_half == 64 ? (size_t)c.n_kv_heads * d * 64 * 2 : 0);
   l.total = o;
   return l;
@@ -167,6 +169,9 @@ struct lola_state {
   bool tensor_path = false;            // bf16, F = 64: tcgen05 kernels
   bool fused_decode = false;           // shapes the one-kernel generation step is built for
   bool have_maps = false;              // TMA descriptors of the sparse cache and the window ring exist
+  bool himg_valid = false;             // the bf16 operand image of H matches H
+  cudaStream_t aux = nullptr;          // second stream: Eq. 10 scoring runs beside the attention kernel
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool force_chain = false;            // set while lola_decode_step_static runs: kernel chain with work lists
   CUtensorMap tm_gk, tm_gv, tm_wk, tm_wv;
   bool profiling = false;
@@ -194,6 +199,16 @@ struct LaunchScope {
   }
 };
 
+template <int DPL>
+int ensure_h_image(lola_state* st, cudaStream_t s) {
+  if (st->himg_valid) return LOLA_OK;
+  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+  k_build_ht_image<DPL><<<st->L.B * st->L.Hkv, 256, 0, s>>>(st->L, (__nv_bfloat16*)(st->base + st->lay.himg));
+  if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
+  st->himg_valid = true;
+  return LOLA_OK;
+}
+
 template <typename T, int DPL>
 int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
@@ -203,10 +218,12 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
     CUtensorMap tq, tk, tv;
     if (make_tokens_map(&tq, c.q, L.B, c.nq, L.Hq, L.d) && make_tokens_map(&tk, c.k, L.B, c.n, L.Hkv, L.d) &&
         make_tokens_map(&tv, c.v, L.B, c.n, L.Hkv, L.d)) {
+      if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
       LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
       dim3 grid2(((L.g + 1) / 2 + 1) / 2, L.B * L.Hkv);
       k_attend2_tc<DPL><<<grid2, kAt2Threads, Attend2Smem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, tq, tk,
-                                                                            tv, (const uint4*)(st->base + st->lay.wt));
+                                                                            tv, (const uint4*)(st->base + st->lay.wt),
+                                                                            (const __nv_bfloat16*)(st->base + st->lay.himg));
       return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
     }
   }
@@ -220,26 +237,37 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
+inline bool fast_update_path(const lola_state* st, const Call& c) {
+  return c.mode == UPD_SELECT && st->have_maps && !st->force_chain && c.count_g % 64 == 0 &&
+         c.r_pos0 + c.r <= c.n_seen && c.count_g + c.r <= kUp2MaxE && c.r <= kUp2MaxFold;
+}
+
 template <typename T, int DPL>
-int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
+int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s, cudaStream_t s_score = nullptr) {
   const Layer& L = st->L;
   const int U = L.B * L.Hkv;
   // chunkwise update on TMA-fed tensor-core kernels: every leaving pair already sits in the ring, the
   // occupied part of the sparse cache is a whole number of 64-slot blocks
-  if (c.mode == UPD_SELECT && st->have_maps && !st->force_chain && c.count_g % 64 == 0 &&
-      c.r_pos0 + c.r <= c.n_seen && c.count_g + c.r <= kUp2MaxE && c.r <= kUp2MaxFold) {
+  if (fast_update_path(st, c)) {
     const int NT = (c.count_g / 64 + (L.eta + 63) / 64 + 1) / 2;
     int tpc = (U * NT + 147) / 148;
     tpc = std::max(2, tpc + (tpc & 1));
     const uint4* img = (const uint4*)(st->base + st->lay.wt);
+    __nv_bfloat16* himg = (__nv_bfloat16*)(st->base + st->lay.himg);
+    if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
     {
-      LaunchScope scope(st, LOLA_KERNEL_SCORE, s);
+      cudaStream_t ss = s_score ? s_score : s;
+      LaunchScope scope(st, LOLA_KERNEL_SCORE, ss);
       dim3 grid((NT + tpc - 1) / tpc, U);
-      k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, tpc);
+      k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
       if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
     }
+    if (s_score) {                       // the selection needs the scores: join the scoring stream
+      if (cudaEventRecord(st->ev_join, s_score) != cudaSuccess || cudaStreamWaitEvent(s, st->ev_join, 0) != cudaSuccess)
+        return LOLA_ERR_CUDA;
+    }
     LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
-    k_update2_tc<DPL><<<U, kUp2Threads, Update2Smem<DPL>::bytes, s>>>(L, c, img);
+    k_update2_tc<DPL><<<U, kUp2Threads, Update2Smem<DPL>::bytes, s>>>(L, c, img, himg);   // keeps the image current
     return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
   }
   if (c.mode == UPD_SELECT) {
@@ -262,6 +290,7 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   }
   LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+  if (c.mode == UPD_SELECT || c.mode == UPD_FOLD_ALL) st->himg_valid = false;   // H changes without its operand image
   k_update<T, DPL><<<U, kUpdThreads, update_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
@@ -269,9 +298,19 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
 template <typename T, int DPL>
 int run_prefill(lola_state* st, Call c, cudaStream_t s) {
   int rc = LOLA_OK;
+  // Attention and scoring both only read the memories: with outputs wanted and the tensor-core update
+  // path in use, the scoring kernel runs on the handle's second stream beside the attention kernel
+  // and the selection joins the two.
+  cudaStream_t s_score = nullptr;
+  if (c.out && st->aux && fast_update_path(st, c)) {
+    if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
+    if (cudaEventRecord(st->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(st->aux, st->ev_fork, 0) != cudaSuccess)
+      return LOLA_ERR_CUDA;
+    s_score = st->aux;
+  }
   if (c.out) rc = launch_attend<T, DPL>(st, c, s);
   if (rc != LOLA_OK) return rc;
-  return launch_update_chain<T, DPL>(st, c, s);
+  return launch_update_chain<T, DPL>(st, c, s, s_score);
 }
 
 template <int DPL>
@@ -291,7 +330,10 @@ template <typename T, int DPL>
 int run_decode(lola_state* st, Call c, cudaStream_t s) {
   // steady state (caches full, one pair leaves the window): the whole step is one kernel
   if (st->fused_decode && !st->force_chain && c.mode == UPD_SELECT && c.r == 1 && c.count_g == st->L.lam)
+  {
+    st->himg_valid = false;              // the fused step folds into H only
     return launch_decode_fused<DPL>(st, c, s);
+  }
   int rc = launch_update_chain<T, DPL>(st, c, s);
   if (rc != LOLA_OK) return rc;
   return launch_attend<T, DPL>(st, c, s);
@@ -388,6 +430,16 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
     }
     for (int i = 0; i < 5; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
   }
+  if (rc == LOLA_OK && st->have_maps) {
+    // host-side objects only (no device memory): a second stream and two events to run the scoring
+    // kernel beside the attention kernel; without them everything stays on the caller's stream
+    if (cudaStreamCreateWithFlags(&st->aux, cudaStreamNonBlocking) != cudaSuccess) st->aux = nullptr;
+    if (st->aux && (cudaEventCreateWithFlags(&st->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                    cudaEventCreateWithFlags(&st->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
+      cudaStreamDestroy(st->aux);
+      st->aux = nullptr;
+    }
+  }
   // one-kernel generation step: lambda a whole number of 64-row blocks, the row stream within 16 tiles
   st->fused_decode = st->have_maps && cfg->sparse >= 64 && cfg->sparse % 64 == 0 && L.g <= kDecQ &&
                      (cfg->sparse / 64 + (cfg->window + 63) / 64 + 1) / 2 <= kDecMaxTiles;
@@ -399,7 +451,7 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
     if (cudaGetLastError() != cudaSuccess) rc = LOLA_ERR_CUDA;
   }
   if (rc == LOLA_OK) rc = lola_reset_state(st, stream);
-  if (rc != LOLA_OK) { delete st; return rc; }
+  if (rc != LOLA_OK) { lola_destroy_state(st); return rc; }
   *out = st;
   return LOLA_OK;
 }
@@ -416,6 +468,7 @@ int lola_reset_state(lola_state* st, void* stream) {
   if (cudaMemsetAsync(L.score, 0xFF, U * ((size_t)c.sparse + c.max_chunk) * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
   if (cudaMemsetAsync(L.thr, 0xFF, U * 2 * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
   st->n_seen = 0;
+  st->himg_valid = true;               // H = 0 and its operand image = 0
   return LOLA_OK;
 }
 
@@ -589,6 +642,7 @@ int lola_write_state(lola_state* st, const lola_state_view* v, void* stream) {
   if (v->threshold) ok = ok && h2d(L.thr, v->threshold, U * 2 * 4);
   if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return LOLA_ERR_CUDA;   // host staging dies here
   st->n_seen = n_seen;
+  st->himg_valid = false;
   return LOLA_OK;
 }
 
@@ -620,6 +674,7 @@ int lola_set_tokens_seen(lola_state* st, int64_t n_seen) {
   if (!st) return LOLA_ERR_ARG;
   if (n_seen < 0 || n_seen > 0x7fffffffLL) return LOLA_ERR_SHAPE;
   st->n_seen = n_seen;
+  st->himg_valid = false;              // the caller replaced the buffer: rebuild H's operand image when needed
   return LOLA_OK;
 }
 
@@ -627,6 +682,9 @@ int lola_destroy_state(lola_state* st) {
   if (!st) return LOLA_ERR_ARG;
   for (auto* v : {&st->records, &st->pool})
     for (ProfRecord& r : *v) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  if (st->aux) { cudaStreamSynchronize(st->aux); cudaStreamDestroy(st->aux); }
+  if (st->ev_fork) cudaEventDestroy(st->ev_fork);
+  if (st->ev_join) cudaEventDestroy(st->ev_join);
   delete st;
   return LOLA_OK;
 }

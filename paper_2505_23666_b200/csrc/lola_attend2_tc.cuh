@@ -12,8 +12,9 @@
 //   warp 8           issues every tcgen05.mma:  S_w = Q_w K^T,  O_w += P_w V  (P_w in tensor memory)
 //   warp 9           TMA producer
 // After the last tile the feature map of the queries is computed (U_w = Q_w W on the tensor cores, one
-// thread per row), scaled by exp(-m) and fed as a tensor-memory A operand into O_w += phi H and into
-// phi [s_hi s_lo], so the linear term lands in the same accumulator and denominator.
+// thread per row), scaled by exp(-m) and fed as a tensor-memory A operand into O_w += phi H (H from its
+// bf16 operand image, bulk-copied at the start), so the linear term lands in the same accumulator; its
+// normaliser exp(-m) phi . s is added to the row's denominator.
 // Every wait on an mbarrier is bounded; a wait that runs out sets bit 64 of the status word and makes
 // the other waits of the CTA return at once.
 #pragma once
@@ -34,35 +35,28 @@ struct Attend2Smem {
   static constexpr uint32_t q = 0;                                   // 2 x [kblk][128][128B]
   static constexpr uint32_t stage0 = 65536;                          // 2 x (K 32 KB + V 32 KB)
   static constexpr uint32_t st_k = 0, st_v = 32768, stage_bytes = 65536;
-  static constexpr uint32_t ht_blk = (d + 16) * 128;
-  static constexpr uint32_t misc = stage0 + 2 * stage_bytes;
+  static constexpr uint32_t ht = stage0 + 2 * stage_bytes;           // H^T operand image [2 j blocks][d][128B]
+  static constexpr uint32_t ht_blk = d * 128;
+  static constexpr uint32_t misc = ht + 32768;
   static constexpr uint32_t total = misc + 1024;
   static constexpr uint32_t bytes = total + 1024;
 };
 
 struct Attend2Misc {
   uint64_t bars[24];
+  float s_vec[128];
   uint32_t tmem_slot;
   int abort_word;
 };
 // barrier indices
-enum { A2_QFULL = 0, A2_KFULL = 1, A2_VFULL = 3, A2_KEMPTY = 5, A2_VEMPTY = 7, A2_SFULL = 9, A2_PREADY = 11, A2_ODONE = 13, A2_WFULL = 15 };
-
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"((uint64_t)(uintptr_t)src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
+enum { A2_QFULL = 0, A2_KFULL = 1, A2_VFULL = 3, A2_KEMPTY = 5, A2_VEMPTY = 7, A2_SFULL = 9, A2_PREADY = 11, A2_ODONE = 13, A2_WFULL = 15, A2_HFULL = 16 };
 
 template <int DPL>
 __global__ void __launch_bounds__(kAt2Threads, 1)
 k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
              const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
              const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_ck,
-             const __grid_constant__ CUtensorMap tm_cv, const uint4* wt_image) {
+             const __grid_constant__ CUtensorMap tm_cv, const uint4* wt_image, const __nv_bfloat16* ht_image) {
   using S = Attend2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
@@ -118,6 +112,8 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   if (warp == 9) {
     // =============================== TMA producer ===============================
     if (lane == 0) {
+      tc::mbar_expect_tx(BAR(A2_HFULL), 2u * d * 128u);
+      tc::bulk_copy_g2s(sbase + S::ht, ht_image + (size_t)unit * (2 * d * 64), 2u * d * 128u, BAR(A2_HFULL));
       // queries: tile w, head slot hs -> rows hs * 64 .. hs * 64 + 63
       tc::mbar_expect_tx(BAR(A2_QFULL), (uint32_t)nw * kblk * 16384u);
       for (int w = 0; w < nw; ++w)
@@ -147,7 +143,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         const int uses = (NT - so + 1) / 2;                       // tiles that went through stage `so`
         if (uses >= 1) ok = WAIT(A2_KEMPTY + so, (uses - 1) & 1) && ok;
         tc::mbar_expect_tx(BAR(A2_WFULL), (uint32_t)kblk * 8192u);
-        bulk_copy_g2s(sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k, wt_image + (size_t)h * kblk * 512, kblk * 8192u,
+        tc::bulk_copy_g2s(sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k, wt_image + (size_t)h * kblk * 512, kblk * 8192u,
                       BAR(A2_WFULL));
       }
       if (!ok) atomicOr(L.status, 64);
@@ -193,12 +189,12 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         if (kt + 1 < NT) tc::mma_commit(BAR(A2_KEMPTY + (st ^ 1)));
       }
       // ---- linear term
-      const int sl = (NT - 1) & 1, so = NT & 1;
+      const int so = NT & 1;
       const uint32_t wt = sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k;
-      const uint32_t ht = sbase + S::stage0 + (uint32_t)sl * S::stage_bytes;
       ok = WAIT(A2_WFULL, 0) && ok;
+      ok = WAIT(A2_HFULL, 0) && ok;
       for (int w = 0; w < nw; ++w) {
-        ok = WAIT(A2_PREADY + w, NT & 1) && ok;                         // H^T staged, S_w free
+        ok = WAIT(A2_PREADY + w, NT & 1) && ok;                         // S_w free
         tc::fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < d / 16; ++ks)
@@ -212,14 +208,10 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         ok = WAIT(A2_PREADY + w, (NT + 1) & 1) && ok;                   // scaled phi(Q_w) in tensor memory
         tc::fence_after_sync();
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint64_t bd = tc::make_desc_sw128(ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024);
-          const uint64_t bs = tc::make_desc_sw128(ht + (ks >> 2) * S::ht_blk + d * 128 + (ks & 3) * 32, 16, 1024);
-          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + 64u + ks * 8, bd,
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + 64u + ks * 8,
+                          tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
                           tc::make_idesc_bf16(128, d, false, false), 1u);
-          tc::mma_bf16_ts(tmem + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + 64u + ks * 8, bs,
-                          tc::make_idesc_bf16(128, 16, false, false), ks > 0);
-        }
         tc::mma_commit(BAR(A2_ODONE + w));
       }
       if (!ok) atomicOr(L.status, 64);
@@ -234,20 +226,8 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     const uint32_t tm_s = tmem + (uint32_t)w * 128u + lane_addr;
     const uint32_t tm_o = tmem + 256u + (uint32_t)w * 128u + lane_addr;
     const int nthr = nw * 128;
-    // H (fp32) for the linear term: with both query tiles active the 256 threads issue the loads now
-    // and convert / store them after the last tile; a lone query tile loads them at the end
-    constexpr int HI = d * (D / 8) / 256;
-    float hreg[HI][8];
-    const float* Hg = L.H + (size_t)unit * D * d;
-    if (nw == 2) {
-#pragma unroll
-      for (int it = 0; it < HI; ++it) {
-        const int i = tid + it * 256;
-        const int cc = i % d, jc = i / d;
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj) hreg[it][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
-      }
-    }
+    if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
+    tc::named_bar_sync(1, nthr);
     float m_used = 0.f, l = 0.f;                       // log2 units; m >= 0 is the stabiliser max(0, max z)
     for (int kt = 0; kt < NT; ++kt) {
       // valid leading columns of each 64-key block of this tile, for this row
@@ -262,25 +242,32 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         else v = 0;
         lim[hb] = max(0, min(64, v));
       }
+      const bool full = lim[0] == 64 && lim[1] == 64;
       ok = WAIT(A2_SFULL + w, kt & 1) && ok;
       tc::fence_after_sync();
+      // pass 1: largest visible score of the row in this tile
       float mx = -CUDART_INF_F;
 #pragma unroll
       for (int c0 = 0; c0 < 128; c0 += 32) {
         float sv[32];
         tc::tmem_ld32(tm_s + c0, sv);
-        const int lm = lim[c0 >> 6] - (c0 & 63);
+        if (full) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, j < lm ? sv[j] : -CUDART_INF_F);
+          for (int j = 0; j < 32; j += 2) mx = fmaxf(mx, fmaxf(sv[j], sv[j + 1]));
+        } else {
+          const int lm = lim[c0 >> 6] - (c0 & 63);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, j < lm ? sv[j] : -CUDART_INF_F);
+        }
       }
       const float m_tile = mx * sl2;
       const bool grow = m_tile > m_used + kGrow;
-      if (__any_sync(0xffffffffu, grow)) {             // rare: rescale what this warp's rows have accumulated
+      if (__any_sync(0xffffffffu, grow)) {             // rare; tensor-memory accesses are warp-wide: every lane takes part
         const float m_new = grow ? m_tile : m_used;
         const float alpha = tc::fast_exp2(m_used - m_new);
         l *= alpha;
         m_used = m_new;
-        if (kt > 0) {                                  // tensor-memory accesses are warp-wide: every lane takes part
+        if (kt > 0) {
           ok = WAIT(A2_ODONE + w, (kt - 1) & 1) && ok;
           tc::fence_after_sync();
 #pragma unroll
@@ -293,19 +280,29 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
           }
         }
       }
+      // pass 2: weights 2^(z - m) <= 2^8, bf16 pairs written over the first half of S
+      float lt = 0.f;
 #pragma unroll
       for (int c0 = 0; c0 < 128; c0 += 32) {
         float sv[32];
         tc::tmem_ld32(tm_s + c0, sv);
-        const int lm = lim[c0 >> 6] - (c0 & 63);
         uint32_t pk[16];
+        if (full) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const float p0 = j < lm ? tc::fast_exp2(fmaf(sv[j], sl2, -m_used)) : 0.f;
-          const float p1 = j + 1 < lm ? tc::fast_exp2(fmaf(sv[j + 1], sl2, -m_used)) : 0.f;
-          const uint32_t pp = pack_bf16x2(p0, p1);
-          l += bf16lo_f(pp) + bf16hi_f(pp);            // the sum uses the weights the product uses
-          pk[j >> 1] = pp;
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = tc::fast_exp2(fmaf(sv[j], sl2, -m_used)), p1 = tc::fast_exp2(fmaf(sv[j + 1], sl2, -m_used));
+            lt += p0 + p1;
+            pk[j >> 1] = pack_bf16x2(p0, p1);
+          }
+        } else {
+          const int lm = lim[c0 >> 6] - (c0 & 63);
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = j < lm ? tc::fast_exp2(fmaf(sv[j], sl2, -m_used)) : 0.f;
+            const float p1 = j + 1 < lm ? tc::fast_exp2(fmaf(sv[j + 1], sl2, -m_used)) : 0.f;
+            lt += p0 + p1;
+            pk[j >> 1] = pack_bf16x2(p0, p1);
+          }
         }
         asm volatile(
             "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n" ::"r"(
@@ -315,56 +312,23 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
             : "memory");
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      l += lt;
       tc::fence_before_sync();
-      mbar_arrive(BAR(A2_PREADY + w));
+      tc::mbar_arrive(BAR(A2_PREADY + w));
     }
-    // ---- linear term: wait for the last PV of this tile, stage H^T over the last tile's stage
+    // ---- linear term: once the last PV of this tile has read P_w, S_w may be overwritten
     ok = WAIT(A2_ODONE + w, (NT - 1) & 1) && ok;
     tc::fence_after_sync();
-    tc::named_bar_sync(1, nthr);                       // both query tiles are done with the last stage
-    {
-      const int sl = (NT - 1) & 1;
-      uint8_t* htp = sm + S::stage0 + (size_t)sl * S::stage_bytes;
-      if (nw == 2) {
-#pragma unroll
-        for (int it = 0; it < HI; ++it) {
-          const int i = tid + it * 256;
-          const int cc = i % d, jc = i / d;
-          *reinterpret_cast<uint4*>(htp + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(hreg[it]);
-        }
-      } else {
-        for (int i = tid; i < d * (D / 8); i += 128) {
-          const int cc = i % d, jc = i / d;
-          float f8[8];
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj) f8[jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
-          *reinterpret_cast<uint4*>(htp + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
-        }
-      }
-      if (tid < D) {
-        const float sv = L.s[(size_t)unit * D + tid];
-        const __nv_bfloat16 hi = __float2bfloat16_rn(sv);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(sv - __bfloat162float(hi));
-        const int ch = (tid & 63) >> 3;
-        *reinterpret_cast<T*>(htp + (tid >> 6) * S::ht_blk + tc::sw128_off(d, ch) + (tid & 7) * 2) = hi;
-        *reinterpret_cast<T*>(htp + (tid >> 6) * S::ht_blk + tc::sw128_off(d + 1, ch) + (tid & 7) * 2) = lo;
-      }
-      for (int i = tid; i < 2 * 14 * 8; i += nthr) {
-        const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
-        *reinterpret_cast<uint4*>(htp + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
-      }
-    }
-    tc::fence_async_smem();
-    tc::fence_before_sync();
-    tc::named_bar_sync(1, nthr);
-    mbar_arrive(BAR(A2_PREADY + w));                   // phase NT: operands staged, S_w may be overwritten
+    tc::mbar_arrive(BAR(A2_PREADY + w));                   // phase NT
     ok = WAIT(A2_SFULL + w, NT & 1) && ok;
     tc::fence_after_sync();
+    float lden = 0.f;                                  // exp(-m) phi(q) . s
     {
       // phi(q) of this row, scaled by exp(-m): bf16 pairs into columns 64..127 of S_w (A operand)
       float u[64];
       tc::tmem_ld64(tm_s, u);
       const float em = tc::fast_exp2(-m_used);
+      float ld0 = 0.f, ld1 = 0.f;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         float e[64];
@@ -388,18 +352,22 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
         uint32_t pk2[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) pk2[i] = pack_bf16x2(e[2 * i] * scale, e[2 * i + 1] * scale);
+        for (int i = 0; i < 32; ++i) {
+          const float f0 = e[2 * i] * scale, f1 = e[2 * i + 1] * scale;
+          ld0 = fmaf(f0, X.s_vec[half * 64 + 2 * i], ld0);
+          ld1 = fmaf(f1, X.s_vec[half * 64 + 2 * i + 1], ld1);
+          pk2[i] = pack_bf16x2(f0, f1);
+        }
         tc::tmem_st32u(tm_s + 64 + half * 32, pk2);
       }
+      lden = ld0 + ld1;
     }
     tc::fence_before_sync();
-    mbar_arrive(BAR(A2_PREADY + w));                   // phase NT + 1
+    tc::mbar_arrive(BAR(A2_PREADY + w));                   // phase NT + 1
     ok = WAIT(A2_ODONE + w, NT & 1) && ok;
     tc::fence_after_sync();
     {
-      float dn[2];
-      tc::tmem_ld2(tm_s, dn);
-      const float inv = 1.0f / (l + dn[0] + dn[1]);
+      const float inv = 1.0f / (l + lden);
       T* op = (T*)c.out + (((size_t)b * n + tok) * L.Hq + h * g + hl) * d;
 #pragma unroll
       for (int c0 = 0; c0 < d; c0 += 32) {

@@ -46,7 +46,7 @@ template <int DPL>
 __global__ void __launch_bounds__(kSc2Threads, 1)
 k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image,
-            int tiles_per_cta) {
+            const __nv_bfloat16* ht_image, int tiles_per_cta) {
   using S = Score2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
@@ -81,7 +81,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   bool ok = true;
 
   if (tid == 0) {
-    for (int i = 0; i < 6; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 8u * i, 1);
+    for (int i = 0; i < 7; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 8u * i, 1);
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
@@ -90,18 +90,16 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile0 + wg, nGB, nRB, unit, bar_k);
     decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile0 + wg, nGB, nRB, unit, bar_v);
   }
-  // ---- operands: H^T (bf16, K-major) with the two parts of s as rows d, d+1; W^T image
+  // ---- operands: H^T operand image (bulk copies, one per j block), the two parts of s as rows d, d+1,
+  //      W^T image
+  const uint32_t bar_h = sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 48u;
+  if (tid == 0) {
+    tc::mbar_expect_tx(bar_h, 2u * d * 128u);
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(ht_image + (size_t)unit * (2 * d * 64));
+    tc::bulk_copy_g2s(sbase + S::ht, src, d * 128u, bar_h);
+    tc::bulk_copy_g2s(sbase + S::ht + S::ht_blk, src + d * 128, d * 128u, bar_h);
+  }
   {
-    constexpr int HI = d * (D / 8) / kSc2Threads;
-    float hreg[HI][8];
-    const float* Hg = L.H + (size_t)unit * D * d;
-#pragma unroll
-    for (int it = 0; it < HI; ++it) {
-      const int i = tid + it * kSc2Threads;
-      const int cc = i % d, jc = i / d;
-#pragma unroll
-      for (int jj = 0; jj < 8; ++jj) hreg[it][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
-    }
     const uint4* img = wt_image + (size_t)h * kblk * 512;
     for (int i = tid; i < kblk * 512; i += kSc2Threads)
       *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
@@ -117,13 +115,8 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
       *reinterpret_cast<uint4*>(sm + S::ht + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
     }
-#pragma unroll
-    for (int it = 0; it < HI; ++it) {
-      const int i = tid + it * kSc2Threads;
-      const int cc = i % d, jc = i / d;
-      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(hreg[it]);
-    }
   }
+  ok = tc::mbar_wait(bar_h, 0) && ok;
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();

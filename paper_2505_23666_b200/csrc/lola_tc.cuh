@@ -143,7 +143,7 @@ __device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier
 
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
   return t;
 }
 
@@ -198,6 +198,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tmap,
 }
 __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)(uintptr_t)tmap) : "memory");
+}
+
+// Linear bulk copy global -> shared (addresses and size multiples of 16 bytes), completion on an mbarrier.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"((uint64_t)(uintptr_t)src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // ---- narrower tensor-memory accesses ------------------------------------------------------------

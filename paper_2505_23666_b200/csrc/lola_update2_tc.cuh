@@ -6,7 +6,7 @@
 //   3. the folded pairs are gathered into operand tiles, phi(K_S) is recomputed
 //      (tcgen05.mma K_S W, feature map with one thread pair per row, rounded to bf16) and
 //      [dH | ds] = phi(K_S)^T [V_S | 1]   (tcgen05.mma, M = 128 features, N = d + 16, K = folded pairs)
-//      is added to H, s with vector reductions at the L2;
+//      is added to H, s; the new H is also written as the bf16 operand image the other kernels load;
 //   4. leaving pairs that stay move into the freed slots; the incoming pairs enter the window ring.
 // Every wait on an mbarrier is bounded; a wait that runs out sets bit 32 of the status word.
 #pragma once
@@ -30,27 +30,31 @@ struct Update2Smem {
   static constexpr uint32_t kt = 16384;                    // K_S tile, K-major [kblk][128][128B]; then phi tile [2][128][128B]
   static constexpr uint32_t vt = kt + 32768;               // [V_S | 1], MN-major: [kblk + 1 column blocks][128 pairs][128B]
   static constexpr uint32_t misc = vt + 3 * 16384;
-  static constexpr uint32_t total = misc + 2 * kUp2MaxE * 4 + 8192;
+  static constexpr uint32_t hs = misc + 2 * kUp2MaxE * 4 + 8192;   // H of the unit, fp32, rows padded by 4 floats
+  static constexpr uint32_t hs_row = (d + 4) * 4;
+  static constexpr uint32_t total = hs + 128 * hs_row;
   static constexpr uint32_t bytes = total + 1024;
 };
 
 struct Update2Misc {
   unsigned key[kUp2MaxE];           // score bits
   int pos[kUp2MaxE];                // position; bit 31 set once the pair is chosen for folding
-  unsigned hist[256];
+  unsigned hist[4][256];
   int scan[kUp2Threads / 32][3];
   int fold_e[kUp2MaxFold];          // E indices of the folded pairs, ascending
   int free_slot[kUp2MaxFold];       // sparse-cache slots of folded members, ascending
   int mover[kUp2MaxFold];           // leaving-pair indices that stay, ascending
-  unsigned sel_prefix, sel_need, min_keep;
-  int n_equal_fold;
+  unsigned min_keep;
+  int n_equal;
+  int equal_e[kUp2MaxFold];         // pairs whose score equals the selection threshold
+  unsigned char fold_mark[kUp2MaxFold];
   uint64_t bars[2];
   uint32_t tmem_slot;
 };
 static_assert(sizeof(Update2Misc) <= 2 * kUp2MaxE * 4 + 8192, "misc region too small");
 
 template <int DPL>
-__global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image) {
+__global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image, __nv_bfloat16* ht_image) {
   using S = Update2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
@@ -72,8 +76,19 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   uint32_t ph = 0;
   bool ok = true;
 
-  if (tid == 0) { tc::mbar_init(bar, 1); tc::mbar_init_fence(); X.min_keep = 0xffffffffu; X.n_equal_fold = 0; }
+  if (tid == 0) { tc::mbar_init(bar, 1); tc::mbar_init_fence(); X.min_keep = 0xffffffffu; X.n_equal = 0; }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
+  // H of the unit streams into shared memory (asynchronous 16-byte copies) while the selection runs
+  {
+    const float* Hg = L.H + (size_t)unit * D * d;
+    for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
+      const int row = i / (d / 4), c4 = i % (d / 4);
+      const uint32_t dst = sbase + S::hs + (uint32_t)row * S::hs_row + (uint32_t)c4 * 16u;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(Hg + (size_t)i * 4) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int i = tid; i < 4 * 256; i += kUp2Threads) (&X.hist[0][0])[i] = 0;
+  }
   // W^T image and zeroed operand tiles can be staged while the selection runs
   {
     const uint4* img = wt_image + (size_t)h * kblk * 512;
@@ -87,20 +102,19 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   }
   // ---- 1. radix select of the nF lowest scores (scores are norms >= 0: bit patterns order like unsigned)
   unsigned prefix = 0, mask = 0, need = (unsigned)nF;
+  __syncthreads();
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    if (tid < 256) X.hist[tid] = 0;
-    __syncthreads();
     for (int e = tid; e < nE; e += kUp2Threads) {
       const unsigned k = X.key[e];
-      if ((k & mask) == prefix) atomicAdd(&X.hist[(k >> shift) & 255u], 1u);
+      if ((k & mask) == prefix) atomicAdd(&X.hist[pass][(k >> shift) & 255u], 1u);
     }
     __syncthreads();
-    if (warp == 0) {
-      // 8 bins per lane, exclusive scan over the 256 bins
+    {
+      // every warp scans the 256 bins itself (8 per lane): no broadcast through shared memory
       unsigned cnt[8], tot = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { cnt[i] = X.hist[lane * 8 + i]; tot += cnt[i]; }
+      for (int i = 0; i < 8; ++i) { cnt[i] = X.hist[pass][lane * 8 + i]; tot += cnt[i]; }
       unsigned incl = tot;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -108,36 +122,57 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
         if (lane >= o) incl += v;
       }
       unsigned run = incl - tot;                     // elements in lower bins
-      if (run < need && need <= incl) {              // exactly one lane holds the bin of the need-th lowest
+      const bool mine = run < need && need <= incl;  // exactly one lane holds the bin of the need-th lowest
+      unsigned np = 0, nn = 0;
+      if (mine) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          if (run < need && need <= run + cnt[i]) {
-            X.sel_prefix = prefix | ((unsigned)(lane * 8 + i) << shift);
-            X.sel_need = need - run;
-          }
+          if (run < need && need <= run + cnt[i]) { np = prefix | ((unsigned)(lane * 8 + i) << shift); nn = need - run; }
           run += cnt[i];
         }
       }
+      const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+      prefix = __shfl_sync(0xffffffffu, np, src);
+      need = __shfl_sync(0xffffffffu, nn, src);
     }
-    __syncthreads();
-    prefix = X.sel_prefix;
-    need = X.sel_need;
     mask |= 255u << shift;
   }
-  // prefix = the nF-th lowest score; `need` of the pairs with exactly that score are folded: the youngest
+  // prefix = the nF-th lowest score; `need` of the pairs with exactly that score are folded: the youngest.
+  // Pairs below the threshold are marked at once; pairs on it are collected into a short list first
+  // (normally one entry) and ranked among themselves by position.
   const unsigned thr_key = prefix;
   for (int e = tid; e < nE; e += kUp2Threads) {
     const unsigned k = X.key[e];
-    bool fold = k < thr_key;
-    if (k == thr_key) {
-      const int pe = X.pos[e] & 0x7fffffff;
-      unsigned younger = 0;
-      for (int j = 0; j < nE; ++j) younger += (X.key[j] == thr_key && (X.pos[j] & 0x7fffffff) > pe) ? 1u : 0u;
-      fold = younger < need;
+    if (k < thr_key) X.pos[e] |= (int)0x80000000;
+    else if (k == thr_key) {
+      const int at = atomicAdd(&X.n_equal, 1);
+      if (at < kUp2MaxFold) X.equal_e[at] = e;
+    } else atomicMin(&X.min_keep, k);
+  }
+  __syncthreads();
+  {
+    const int neq = X.n_equal;
+    if (neq <= kUp2MaxFold) {
+      for (int i = tid; i < neq; i += kUp2Threads) {
+        const int e = X.equal_e[i], pe = X.pos[e];
+        unsigned younger = 0;
+        for (int j = 0; j < neq; ++j) younger += X.pos[X.equal_e[j]] > pe ? 1u : 0u;
+        if (younger < need) X.fold_mark[i] = 1; else { X.fold_mark[i] = 0; atomicMin(&X.min_keep, thr_key); }
+      }
+      __syncthreads();
+      for (int i = tid; i < neq; i += kUp2Threads)
+        if (X.fold_mark[i]) X.pos[X.equal_e[i]] |= (int)0x80000000;
+    } else {
+      // many equal scores (degenerate inputs): rank every one of them against all pairs
+      for (int e = tid; e < nE; e += kUp2Threads) {
+        if (X.key[e] != thr_key) continue;
+        const int pe = X.pos[e] & 0x7fffffff;
+        unsigned younger = 0;
+        for (int j = 0; j < nE; ++j) younger += (X.key[j] == thr_key && (X.pos[j] & 0x7fffffff) > pe) ? 1u : 0u;
+        if (younger < need) atomicOr(reinterpret_cast<unsigned*>(&X.pos[e]), 0x80000000u);
+        else atomicMin(&X.min_keep, thr_key);
+      }
     }
-    if (!fold) atomicMin(&X.min_keep, k);
-    // mark (other threads read pos only through the 31-bit mask above)
-    if (fold) atomicOr(reinterpret_cast<unsigned*>(&X.pos[e]), 0x80000000u);
   }
   __syncthreads();
   // ---- 2. ordered compaction: each thread owns a contiguous range of E
@@ -246,6 +281,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
       *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t, ch)) = o;
     }
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
@@ -262,23 +298,45 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1;
   tc::fence_after_sync();
   if (tid < 256 && ok) {                                             // row j = t, columns [hf * d/2, +d/2)
+    // H += dH in the shared-memory copy (this thread owns the half row) and the same values as bf16 in
+    // the operand image layout [2 j blocks][d rows c][64 j] (row c, K index j, 128-byte swizzle), staged
+    // over the consumed phi tile; both leave through coalesced stores below
     constexpr int HC = d / 2;
-    float* Hrow = L.H + ((size_t)unit * D + t) * d + hf * HC;
+    float* Hrow = reinterpret_cast<float*>(sm + S::hs + (size_t)t * S::hs_row) + hf * HC;
+    const uint32_t joff = (uint32_t)(t >> 6) * (d * 128) + (uint32_t)(t & 7) * 2;
+    const int jch = (t & 63) >> 3;
 #pragma unroll
     for (int c0 = 0; c0 < HC; c0 += 32) {
       float p[32];
       tc::tmem_ld32(tm_d + lane_addr + hf * HC + c0, p);
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Hrow + c0 + q * 4), "f"(p[q * 4]), "f"(p[q * 4 + 1]),
-                     "f"(p[q * 4 + 2]), "f"(p[q * 4 + 3])
-                     : "memory");
+      for (int q = 0; q < 8; ++q) {
+        float4 hv = *reinterpret_cast<const float4*>(Hrow + c0 + q * 4);
+        hv.x += p[q * 4]; hv.y += p[q * 4 + 1]; hv.z += p[q * 4 + 2]; hv.w += p[q * 4 + 3];
+        *reinterpret_cast<float4*>(Hrow + c0 + q * 4) = hv;
+        p[q * 4] = hv.x; p[q * 4 + 1] = hv.y; p[q * 4 + 2] = hv.z; p[q * 4 + 3] = hv.w;
+      }
+#pragma unroll
+      for (int q = 0; q < 32; ++q) {
+        const int cc = hf * HC + c0 + q;
+        *reinterpret_cast<__nv_bfloat16*>(sm + S::kt + joff + tc::sw128_off(cc, jch)) = __float2bfloat16_rn(p[q]);
+      }
     }
     if (hf == 0) {
       float ds[2];
       tc::tmem_ld2(tm_d + lane_addr + d, ds);
-      atomicAdd(L.s + (size_t)unit * D + t, ds[0]);
+      L.s[(size_t)unit * D + t] += ds[0];
     }
+  }
+  __syncthreads();
+  if (ok) {
+    float4* Hg4 = reinterpret_cast<float4*>(L.H + (size_t)unit * D * d);
+    for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
+      const int row = i / (d / 4), c4 = i % (d / 4);
+      Hg4[i] = *reinterpret_cast<const float4*>(sm + S::hs + (size_t)row * S::hs_row + (size_t)c4 * 16);
+    }
+    uint4* img4 = reinterpret_cast<uint4*>(ht_image + (size_t)unit * (2 * d * 64));
+    for (int i = tid; i < 2 * d * 128 / 16; i += kUp2Threads) img4[i] = *reinterpret_cast<const uint4*>(sm + S::kt + (size_t)i * 16);
   }
   // ---- 4. leaving pairs that stay: into the freed slots, then into the slots beyond count_g
   for (int i = tid; i < nMove * nch * 2; i += kUp2Threads) {
@@ -313,6 +371,23 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tmem, 256);
+}
+
+// Rebuilds the bf16 operand image of H for every unit (after a path that changed H without
+// maintaining it): per unit [2 j blocks][d rows c][64 j], 128-byte swizzle.
+template <int DPL>
+__global__ void __launch_bounds__(256) k_build_ht_image(Layer L, __nv_bfloat16* ht_image) {
+  constexpr int d = DPL * 32, D = 128;
+  const int unit = blockIdx.x;
+  const float* Hg = L.H + (size_t)unit * D * d;
+  uint8_t* img = reinterpret_cast<uint8_t*>(ht_image + (size_t)unit * (2 * d * 64));
+  for (int i = threadIdx.x; i < d * (D / 8); i += 256) {
+    const int cc = i % d, jc = i / d;
+    float f8[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) f8[jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+    *reinterpret_cast<uint4*>(img + (jc >> 3) * (d * 128) + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
+  }
 }
 
 }  // namespace lola

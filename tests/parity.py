@@ -44,16 +44,17 @@ def close(gpu: np.ndarray, ref: np.ndarray, tol: float, kind: str):
 
 class Lockstep:
     def __init__(self, wl: Workload, rows=None, threads: int = 8, device="cuda:0", inputs: WorkloadInputs = None,
-                 generic_kernels: bool = False):
+                 generic_kernels: bool = False, softmax_scale: float = 0.0):
         self.wl = wl
         self.rows = list(range(wl.batch)) if rows is None else list(rows)
         self.inputs = inputs or WorkloadInputs(wl)
         B = len(self.rows)
         self.tol = tolerances(wl.dtype)
-        self.ocfg = config_for(wl, batch=B)
+        self.ocfg = config_for(wl, batch=B, softmax_scale=(softmax_scale or None))
         self.oracle = LolaOracle(self.ocfg, self.inputs.W.astype(np.float64), threads=threads)
         self.cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window,
-                                       wl.sparse, max(wl.chunk, 1), dtype=wl.dtype, generic_kernels=generic_kernels)
+                                       wl.sparse, max(wl.chunk, 1), dtype=wl.dtype, generic_kernels=generic_kernels,
+                                       softmax_scale=softmax_scale)
         self.layer = binding.LolaLayer(self.cfg, self.inputs.W, device=device)
         self.resyncs = 0
         self.scored_updates = 0

@@ -86,6 +86,17 @@ def test_cfg3_shape_decode_sample():
     assert summ["resyncs"] <= 2, summ
 
 
+@pytest.mark.parametrize("scale", [0.7, 3.0])
+def test_large_logits_move_the_stabiliser(scale):
+    """A softmax scale far above 1/sqrt(d) makes q.k exceed the stabiliser by many powers of two inside
+    a tile, so the attention kernels must rescale what they have accumulated (sums, weights, outputs)."""
+    wl = small_case("hot", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=448, chunk=64,
+                    window=64, sparse=192, dtype="bf16", seed=17, decode_steps=6)
+    ls = Lockstep(wl, threads=1, softmax_scale=scale)
+    summ = drive(ls, 448, 64, 6)
+    assert summ["resyncs"] <= 2, summ
+
+
 def test_bf16_generic_kernels_flag():
     """The CUDA-core kernels stay available in bf16 mode behind a config flag and meet the same bar."""
     wl = small_case("bf16_generic", batch=2, n_q_heads=4, n_kv_heads=2, head_dim=128, feat_half=64, tokens=200,
