@@ -242,33 +242,50 @@ inline bool fast_update_path(const lola_state* st, const Call& c) {
          c.r_pos0 + c.r <= c.n_seen && c.count_g + c.r <= kUp2MaxE && c.r <= kUp2MaxFold;
 }
 
+// Eq. 10 scoring and the top-lambda selection on TMA-fed tensor-core kernels.  Both only read the
+// memories (scores, positions) and write scores / work lists, so they may run beside the attention
+// kernel on another stream.
+template <int DPL>
+int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss) {
+  const Layer& L = st->L;
+  const int U = L.B * L.Hkv;
+  const int NT = (c.count_g / 64 + (L.eta + 63) / 64 + 1) / 2;
+  int tpc = (U * NT + 147) / 148;
+  tpc = std::max(2, tpc + (tpc & 1));
+  const uint4* img = (const uint4*)(st->base + st->lay.wt);
+  __nv_bfloat16* himg = (__nv_bfloat16*)(st->base + st->lay.himg);
+  {
+    LaunchScope scope(st, LOLA_KERNEL_SCORE, ss);
+    dim3 grid((NT + tpc - 1) / tpc, U);
+    k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
+    if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
+  }
+  LaunchScope scope(st, LOLA_KERNEL_SELECT, ss);
+  k_update2_tc<DPL, 1><<<U, kUp2Threads, sizeof(Update2Misc) + 1024, ss>>>(L, c, img, himg);
+  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
+// Eq. 13 fold, moves into the sparse cache and window roll from the selection's work lists; keeps the
+// operand image of H current.
+template <int DPL>
+int launch_apply(lola_state* st, const Call& c, cudaStream_t s) {
+  const Layer& L = st->L;
+  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+  k_update2_tc<DPL, 2><<<L.B * L.Hkv, kUp2Threads, Update2Smem<DPL>::bytes, s>>>(
+      L, c, (const uint4*)(st->base + st->lay.wt), (__nv_bfloat16*)(st->base + st->lay.himg));
+  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
 template <typename T, int DPL>
-int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s, cudaStream_t s_score = nullptr) {
+int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   const int U = L.B * L.Hkv;
   // chunkwise update on TMA-fed tensor-core kernels: every leaving pair already sits in the ring, the
   // occupied part of the sparse cache is a whole number of 64-slot blocks
   if (fast_update_path(st, c)) {
-    const int NT = (c.count_g / 64 + (L.eta + 63) / 64 + 1) / 2;
-    int tpc = (U * NT + 147) / 148;
-    tpc = std::max(2, tpc + (tpc & 1));
-    const uint4* img = (const uint4*)(st->base + st->lay.wt);
-    __nv_bfloat16* himg = (__nv_bfloat16*)(st->base + st->lay.himg);
     if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
-    {
-      cudaStream_t ss = s_score ? s_score : s;
-      LaunchScope scope(st, LOLA_KERNEL_SCORE, ss);
-      dim3 grid((NT + tpc - 1) / tpc, U);
-      k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
-      if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
-    }
-    if (s_score) {                       // the selection needs the scores: join the scoring stream
-      if (cudaEventRecord(st->ev_join, s_score) != cudaSuccess || cudaStreamWaitEvent(s, st->ev_join, 0) != cudaSuccess)
-        return LOLA_ERR_CUDA;
-    }
-    LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
-    k_update2_tc<DPL><<<U, kUp2Threads, Update2Smem<DPL>::bytes, s>>>(L, c, img, himg);   // keeps the image current
-    return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+    int rc = launch_score_select<DPL>(st, c, s);
+    return rc == LOLA_OK ? launch_apply<DPL>(st, c, s) : rc;
   }
   if (c.mode == UPD_SELECT) {
     const int nE = c.count_g + c.r;
@@ -301,16 +318,23 @@ int run_prefill(lola_state* st, Call c, cudaStream_t s) {
   // Attention and scoring both only read the memories: with outputs wanted and the tensor-core update
   // path in use, the scoring kernel runs on the handle's second stream beside the attention kernel
   // and the selection joins the two.
-  cudaStream_t s_score = nullptr;
   if (c.out && st->aux && fast_update_path(st, c)) {
     if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
     if (cudaEventRecord(st->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(st->aux, st->ev_fork, 0) != cudaSuccess)
       return LOLA_ERR_CUDA;
-    s_score = st->aux;
+    // scoring and selection are enqueued first: their many short CTAs take the SMs at once and the
+    // attention CTAs fill in as they drain; the fold joins both
+    rc = launch_score_select<DPL>(st, c, st->aux);
+    if (rc != LOLA_OK) return rc;
+    rc = launch_attend<T, DPL>(st, c, s);
+    if (rc != LOLA_OK) return rc;
+    if (cudaEventRecord(st->ev_join, st->aux) != cudaSuccess || cudaStreamWaitEvent(s, st->ev_join, 0) != cudaSuccess)
+      return LOLA_ERR_CUDA;
+    return launch_apply<DPL>(st, c, s);
   }
   if (c.out) rc = launch_attend<T, DPL>(st, c, s);
   if (rc != LOLA_OK) return rc;
-  return launch_update_chain<T, DPL>(st, c, s, s_score);
+  return launch_update_chain<T, DPL>(st, c, s);
 }
 
 template <int DPL>
@@ -419,13 +443,13 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       e[0] = cudaFuncSetAttribute(k_decode_tc<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
       e[1] = cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
       e[2] = cudaFuncSetAttribute(k_score2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<4>::bytes);
-      e[3] = cudaFuncSetAttribute(k_update2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<4>::bytes);
+      e[3] = cudaFuncSetAttribute(k_update2_tc<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<4>::bytes);
       e[4] = cudaFuncSetAttribute(k_attend2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<4>::bytes);
     } else {
       e[0] = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[1] = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[2] = cudaFuncSetAttribute(k_score2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<2>::bytes);
-      e[3] = cudaFuncSetAttribute(k_update2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<2>::bytes);
+      e[3] = cudaFuncSetAttribute(k_update2_tc<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<2>::bytes);
       e[4] = cudaFuncSetAttribute(k_attend2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<2>::bytes);
     }
     for (int i = 0; i < 5; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape

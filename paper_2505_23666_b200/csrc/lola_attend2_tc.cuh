@@ -6,11 +6,11 @@
 // 64 token slots.  Keys and values stream through two shared-memory stages in tiles of 128 rows
 // (64-row blocks of sparse-cache slots, ring slots, then the incoming chunk), loaded once for both
 // query tiles by TMA.  Warp roles:
-//   warps 0-3 / 4-7  softmax of query tile 0 / 1, one thread per row: S from tensor memory, masked
+//   warps 0-7 / 8-15 softmax of query tile 0 / 1, two threads per row (64 keys each): S from tensor memory, masked
 //                    maximum (the stabiliser only moves when it must grow by more than 2^8), weights
 //                    exp(z - m) rounded to bf16 and written back over S as the A operand of PV
-//   warp 8           issues every tcgen05.mma:  S_w = Q_w K^T,  O_w += P_w V  (P_w in tensor memory)
-//   warp 9           TMA producer
+//   warp 16          issues every tcgen05.mma:  S_w = Q_w K^T,  O_w += P_w V  (P_w in tensor memory)
+//   warp 17          TMA producer
 // After the last tile the feature map of the queries is computed (U_w = Q_w W on the tensor cores, one
 // thread per row), scaled by exp(-m) and fed as a tensor-memory A operand into O_w += phi H (H from its
 // bf16 operand image, bulk-copied at the start), so the linear term lands in the same accumulator; its
@@ -26,7 +26,7 @@
 
 namespace lola {
 
-constexpr int kAt2Threads = 320;
+constexpr int kAt2Threads = 576;
 
 template <int DPL>
 struct Attend2Smem {
@@ -38,13 +38,15 @@ struct Attend2Smem {
   static constexpr uint32_t ht = stage0 + 2 * stage_bytes;           // H^T operand image [2 j blocks][d][128B]
   static constexpr uint32_t ht_blk = d * 128;
   static constexpr uint32_t misc = ht + 32768;
-  static constexpr uint32_t total = misc + 1024;
-  static constexpr uint32_t bytes = total + 1024;
+  static constexpr uint32_t total = misc + 2816;
+  static constexpr uint32_t bytes = 232448;                          // all of an SM's shared memory; the base is aligned at run time
 };
 
 struct Attend2Misc {
   uint64_t bars[24];
   float s_vec[128];
+  float hx[2][2][128];           // [query tile][half][row]: row maxima of the two halves of a key tile; at the end
+                                 // the two halves of the row's denominator
   uint32_t tmem_slot;
   int abort_word;
 };
@@ -74,6 +76,10 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   auto WAIT = [&](int i, uint32_t parity) { return tc::mbar_wait(BAR(i), parity, abortw); };
 
   if (*reinterpret_cast<volatile int*>(L.status) != 0) return;     // an earlier kernel failed: do nothing
+  if ((uint32_t)(sm - smem_raw) + S::total > S::bytes) {            // (cannot happen with a 1024-byte aligned window)
+    if (threadIdx.x == 0) atomicOr(L.status, 64);
+    return;
+  }
 
   const int unit = blockIdx.y, b = unit / L.Hkv, h = unit % L.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -88,7 +94,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
 
   if (tid == 0) {
     X.abort_word = 0;
-    for (int i = 0; i < 17; ++i) tc::mbar_init(BAR(i), (i == A2_PREADY || i == A2_PREADY + 1) ? 128u : 1u);
+    for (int i = 0; i < 17; ++i) tc::mbar_init(BAR(i), (i == A2_PREADY || i == A2_PREADY + 1) ? 256u : 1u);
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
@@ -109,7 +115,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
   };
 
-  if (warp == 9) {
+  if (warp == 17) {
     // =============================== TMA producer ===============================
     if (lane == 0) {
       tc::mbar_expect_tx(BAR(A2_HFULL), 2u * d * 128u);
@@ -148,7 +154,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       }
       if (!ok) atomicOr(L.status, 64);
     }
-  } else if (warp == 8) {
+  } else if (warp == 16) {
     // =============================== MMA issuer ===============================
     if (lane == 0) {
       const uint32_t idesc_s = tc::make_idesc_bf16(128, 128, false, false);
@@ -166,7 +172,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         const uint32_t stage = sbase + S::stage0 + (uint32_t)(kt & 1) * S::stage_bytes;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + ks * 8,
+          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + (uint32_t)(ks >> 2) * 64u + (ks & 3) * 8,
                           tc::make_desc_sw128(stage + S::st_v + ks * 2048, 16384, 1024), idesc_pv, (kt > 0 || ks > 0) ? 1u : 0u);
         tc::mma_commit(BAR(A2_ODONE + w));
       };
@@ -216,51 +222,51 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       }
       if (!ok) atomicOr(L.status, 64);
     }
-  } else if (warp < 4 * nw) {
-    // =============================== softmax, one thread per query row ===============================
-    const int w = warp >> 2, wq = warp & 3;
+  } else if (warp < 8 * nw) {
+    // =============================== softmax, two threads per query row ===============================
+    // thread (query tile w, row t, half hf) owns the 64 keys [64 hf, 64 hf + 64) of every key tile, half of
+    // the feature map in the linear term and half of the output columns
+    const int w = warp >> 3, hf = (warp >> 2) & 1, wq = warp & 3;
     const int t = wq * 32 + lane;                      // row of the query tile = tensor-memory lane
     const int hl = (qt0 + w) * 2 + (t >> 6), tok = t & 63;
     const bool row_ok = hl < g && tok < n;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const uint32_t tm_s = tmem + (uint32_t)w * 128u + lane_addr;
+    const uint32_t tm_sb = tm_s + (uint32_t)hf * 64u;  // this thread's 64 score columns; its weights go to the first 32
     const uint32_t tm_o = tmem + 256u + (uint32_t)w * 128u + lane_addr;
-    const int nthr = nw * 128;
+    constexpr int HC = d / 2;
     if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
-    tc::named_bar_sync(1, nthr);
     float m_used = 0.f, l = 0.f;                       // log2 units; m >= 0 is the stabiliser max(0, max z)
     for (int kt = 0; kt < NT; ++kt) {
-      // valid leading columns of each 64-key block of this tile, for this row
-      int lim[2];
-#pragma unroll
-      for (int hb = 0; hb < 2; ++hb) {
-        const int blk = 2 * kt + hb;
-        int v;
-        if (blk < nGB) v = att_g - blk * 64;
-        else if (blk < nGB + nRB) v = cw - (blk - nGB) * 64;
-        else if (blk == nGB + nRB) v = min(n, tok + 1);
-        else v = 0;
-        lim[hb] = max(0, min(64, v));
-      }
-      const bool full = lim[0] == 64 && lim[1] == 64;
+      // valid leading columns of this thread's 64-key block of the tile, for this row
+      const int blk = 2 * kt + hf;
+      int lim;
+      if (blk < nGB) lim = att_g - blk * 64;
+      else if (blk < nGB + nRB) lim = cw - (blk - nGB) * 64;
+      else if (blk == nGB + nRB) lim = min(n, tok + 1);
+      else lim = 0;
+      lim = max(0, min(64, lim));
       ok = WAIT(A2_SFULL + w, kt & 1) && ok;
       tc::fence_after_sync();
-      // pass 1: largest visible score of the row in this tile
-      float mx = -CUDART_INF_F;
+      float sv[64];
+      tc::tmem_ld64(tm_sb, sv);
+      float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+      if (lim == 64) {
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        float sv[32];
-        tc::tmem_ld32(tm_s + c0, sv);
-        if (full) {
+        for (int j = 0; j < 64; j += 4) {
+          mx0 = fmaxf(mx0, fmaxf(sv[j], sv[j + 1]));
+          mx1 = fmaxf(mx1, fmaxf(sv[j + 2], sv[j + 3]));
+        }
+      } else {
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) mx = fmaxf(mx, fmaxf(sv[j], sv[j + 1]));
-        } else {
-          const int lm = lim[c0 >> 6] - (c0 & 63);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, j < lm ? sv[j] : -CUDART_INF_F);
+        for (int j = 0; j < 64; ++j) {
+          sv[j] = j < lim ? sv[j] : -CUDART_INF_F;     // masked keys get weight 2^(-inf) = 0 below
+          mx0 = fmaxf(mx0, sv[j]);
         }
       }
-      const float m_tile = mx * sl2;
+      X.hx[w][hf][t] = fmaxf(mx0, mx1);
+      tc::named_bar_sync(1 + w, 256);                  // (also: both halves hold their scores in registers now)
+      const float m_tile = fmaxf(X.hx[w][0][t], X.hx[w][1][t]) * sl2;
       const bool grow = m_tile > m_used + kGrow;
       if (__any_sync(0xffffffffu, grow)) {             // rare; tensor-memory accesses are warp-wide: every lane takes part
         const float m_new = grow ? m_tile : m_used;
@@ -271,108 +277,107 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
           ok = WAIT(A2_ODONE + w, (kt - 1) & 1) && ok;
           tc::fence_after_sync();
 #pragma unroll
-          for (int c0 = 0; c0 < d; c0 += 8) {
+          for (int c0 = 0; c0 < HC; c0 += 8) {         // this thread's half of the row's output columns
             float ov[8];
-            tc::tmem_ld8(tm_o + c0, ov);
+            tc::tmem_ld8(tm_o + hf * HC + c0, ov);
 #pragma unroll
             for (int j = 0; j < 8; ++j) ov[j] *= alpha;
-            tc::tmem_st8(tm_o + c0, ov);
+            tc::tmem_st8(tm_o + hf * HC + c0, ov);
           }
         }
       }
-      // pass 2: weights 2^(z - m) <= 2^8, bf16 pairs written over the first half of S
-      float lt = 0.f;
+      // weights 2^(z - m) <= 2^8 as bf16 pairs over the first half of this thread's S columns
+      float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        float sv[32];
-        tc::tmem_ld32(tm_s + c0, sv);
+      for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t pk[16];
-        if (full) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = tc::fast_exp2(fmaf(sv[j], sl2, -m_used)), p1 = tc::fast_exp2(fmaf(sv[j + 1], sl2, -m_used));
-            lt += p0 + p1;
-            pk[j >> 1] = pack_bf16x2(p0, p1);
-          }
-        } else {
-          const int lm = lim[c0 >> 6] - (c0 & 63);
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = j < lm ? tc::fast_exp2(fmaf(sv[j], sl2, -m_used)) : 0.f;
-            const float p1 = j + 1 < lm ? tc::fast_exp2(fmaf(sv[j + 1], sl2, -m_used)) : 0.f;
-            lt += p0 + p1;
-            pk[j >> 1] = pack_bf16x2(p0, p1);
-          }
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = tc::fast_exp2(fmaf(sv[c0 + j], sl2, -m_used)), p1 = tc::fast_exp2(fmaf(sv[c0 + j + 1], sl2, -m_used));
+          l0 += p0;
+          l1 += p1;
+          pk[j >> 1] = pack_bf16x2(p0, p1);
         }
         asm volatile(
             "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n" ::"r"(
-                tm_s + (c0 >> 1)),
+                tm_sb + (c0 >> 1)),
             "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]), "r"(pk[8]), "r"(pk[9]),
             "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
             : "memory");
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-      l += lt;
+      l += l0 + l1;
       tc::fence_before_sync();
       tc::mbar_arrive(BAR(A2_PREADY + w));
     }
     // ---- linear term: once the last PV of this tile has read P_w, S_w may be overwritten
     ok = WAIT(A2_ODONE + w, (NT - 1) & 1) && ok;
     tc::fence_after_sync();
-    tc::mbar_arrive(BAR(A2_PREADY + w));                   // phase NT
+    tc::mbar_arrive(BAR(A2_PREADY + w));               // phase NT
     ok = WAIT(A2_SFULL + w, NT & 1) && ok;
     tc::fence_after_sync();
-    float lden = 0.f;                                  // exp(-m) phi(q) . s
+    float lden = 0.f;                                  // the other half of the row's denominator
     {
-      // phi(q) of this row, scaled by exp(-m): bf16 pairs into columns 64..127 of S_w (A operand)
-      float u[64];
-      tc::tmem_ld64(tm_s, u);
+      // this thread's half of phi(q) (hf = 0: softmax(u), 1: softmax(-u)), scaled by exp(-m): bf16 pairs
+      // into columns 64 + 32 hf .. of S_w (A operand of the linear product)
+      float e[64];
+      tc::tmem_ld64(tm_s, e);
       const float em = tc::fast_exp2(-m_used);
+      const float sgn = hf ? -kLog2e : kLog2e;
+      float scale;
+      if (L.phi_kind == 1) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
+        scale = em;
+      } else {
+        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) { m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn); }
+        const float mm = fmaxf(m0, m1);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) {
+          e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
+          e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
+        }
+        scale = em / (s0 + s1);
+      }
       float ld0 = 0.f, ld1 = 0.f;
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float e[64];
-        const float sgn = half ? -kLog2e : kLog2e;
-        float scale;
-        if (L.phi_kind == 1) {
-#pragma unroll
-          for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(u[i] * sgn);
-          scale = em;
-        } else {
-          float mm = -CUDART_INF_F;
-#pragma unroll
-          for (int i = 0; i < 64; ++i) mm = fmaxf(mm, u[i] * sgn);
-          float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-          for (int i = 0; i < 64; i += 2) {
-            e[i] = tc::fast_exp2(fmaf(u[i], sgn, -mm)); s0 += e[i];
-            e[i + 1] = tc::fast_exp2(fmaf(u[i + 1], sgn, -mm)); s1 += e[i + 1];
-          }
-          scale = em / (s0 + s1);
-        }
-        uint32_t pk2[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float f0 = e[2 * i] * scale, f1 = e[2 * i + 1] * scale;
-          ld0 = fmaf(f0, X.s_vec[half * 64 + 2 * i], ld0);
-          ld1 = fmaf(f1, X.s_vec[half * 64 + 2 * i + 1], ld1);
-          pk2[i] = pack_bf16x2(f0, f1);
-        }
-        tc::tmem_st32u(tm_s + 64 + half * 32, pk2);
+      for (int i = 0; i < 64; i += 2) {
+        e[i] *= scale;
+        e[i + 1] *= scale;
+        ld0 = fmaf(e[i], X.s_vec[hf * 64 + i], ld0);
+        ld1 = fmaf(e[i + 1], X.s_vec[hf * 64 + i + 1], ld1);
       }
-      lden = ld0 + ld1;
+      X.hx[w][hf][t] = l + ld0 + ld1;
+      tc::named_bar_sync(1 + w, 256);                  // both halves have read U before columns 64.. are overwritten
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) pk[j >> 1] = pack_bf16x2(e[c0 + j], e[c0 + j + 1]);
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n" ::"r"(
+                tm_s + 64 + hf * 32 + (c0 >> 1)),
+            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]), "r"(pk[8]), "r"(pk[9]),
+            "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
+            : "memory");
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      lden = X.hx[w][hf ^ 1][t];
     }
     tc::fence_before_sync();
-    tc::mbar_arrive(BAR(A2_PREADY + w));                   // phase NT + 1
+    tc::mbar_arrive(BAR(A2_PREADY + w));               // phase NT + 1
     ok = WAIT(A2_ODONE + w, NT & 1) && ok;
     tc::fence_after_sync();
     {
-      const float inv = 1.0f / (l + lden);
-      T* op = (T*)c.out + (((size_t)b * n + tok) * L.Hq + h * g + hl) * d;
+      const float inv = 1.0f / (X.hx[w][hf][t] + lden);
+      T* op = (T*)c.out + (((size_t)b * n + tok) * L.Hq + h * g + hl) * d + hf * HC;
 #pragma unroll
-      for (int c0 = 0; c0 < d; c0 += 32) {
+      for (int c0 = 0; c0 < HC; c0 += 32) {
         float ov[32];
-        tc::tmem_ld32(tm_o + c0, ov);
+        tc::tmem_ld32(tm_o + hf * HC + c0, ov);
         if (row_ok && ok) {
 #pragma unroll
           for (int q8 = 0; q8 < 4; ++q8) {
@@ -386,7 +391,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
       }
     }
-    if (!ok && t == 0) atomicOr(L.status, 64);
+    if (!ok && t == 0 && hf == 0) atomicOr(L.status, 64);
   }
   tc::fence_before_sync();
   __syncthreads();

@@ -53,7 +53,9 @@ struct Update2Misc {
 };
 static_assert(sizeof(Update2Misc) <= 2 * kUp2MaxE * 4 + 8192, "misc region too small");
 
-template <int DPL>
+// PHASE 1: selection only (steps 1-2; the lists go to the state's work-list arrays, so it can run beside
+// the attention kernel, which only reads the memories).  PHASE 2: steps 3-4 from those lists.
+template <int DPL, int PHASE>
 __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image, __nv_bfloat16* ht_image) {
   using S = Update2Smem<DPL>;
   constexpr int d = DPL * 32;
@@ -65,21 +67,26 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = tc::smem_u32(sm);
-  Update2Misc& X = *reinterpret_cast<Update2Misc*>(sm + S::misc);
+  constexpr uint32_t kMisc = PHASE == 1 ? 0u : S::misc;          // the selection needs the small arrays only
+  Update2Misc& X = *reinterpret_cast<Update2Misc*>(sm + kMisc);
 
   const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lam = L.lam, eta = L.eta;
   const int cg = c.count_g, nE = cg + c.r, nF = nE - lam;          // 1 <= nF <= min(r, kUp2MaxFold)
   float* scu = L.score + (size_t)unit * (lam + L.cmax);
-  const uint32_t bar = sbase + S::misc + (uint32_t)offsetof(Update2Misc, bars);
+  const uint32_t bar = sbase + kMisc + (uint32_t)offsetof(Update2Misc, bars);
+  int* g_fold = L.fold_idx + (size_t)unit * L.cmax;
+  int* g_src = L.move_src + (size_t)unit * L.cmax;
+  int* g_dst = L.move_dst + (size_t)unit * L.cmax;
+  int* g_cnt = L.counts + (size_t)unit * 4;
   uint32_t ph = 0;
   bool ok = true;
 
   if (tid == 0) { tc::mbar_init(bar, 1); tc::mbar_init_fence(); X.min_keep = 0xffffffffu; X.n_equal = 0; }
-  if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
-  // H of the unit streams into shared memory (asynchronous 16-byte copies) while the selection runs
-  {
+  if (PHASE != 1 && warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
+  // H of the unit streams into shared memory (asynchronous 16-byte copies) meanwhile
+  if (PHASE != 1) {
     const float* Hg = L.H + (size_t)unit * D * d;
     for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
       const int row = i / (d / 4), c4 = i % (d / 4);
@@ -87,15 +94,19 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(Hg + (size_t)i * 4) : "memory");
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int i = tid; i < 4 * 256; i += kUp2Threads) (&X.hist[0][0])[i] = 0;
   }
-  // W^T image and zeroed operand tiles can be staged while the selection runs
-  {
+  if (PHASE != 2)
+    for (int i = tid; i < 4 * 256; i += kUp2Threads) (&X.hist[0][0])[i] = 0;
+  // W^T image and zeroed operand tiles
+  if (PHASE != 1) {
     const uint4* img = wt_image + (size_t)h * kblk * 512;
     for (int i = tid; i < kblk * 512; i += kUp2Threads) *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
     for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
       *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
   }
+  int nGL = 0, nMove = 0;
+  unsigned thr_key = 0;
+  if (PHASE != 2) {
   for (int e = tid; e < nE; e += kUp2Threads) {
     if (e < cg) { X.key[e] = __float_as_uint(scu[e]); X.pos[e] = L.gpos[(size_t)unit * lam + e]; }
     else { X.key[e] = __float_as_uint(scu[lam + (e - cg)]); X.pos[e] = c.r_pos0 + (e - cg); }
@@ -140,7 +151,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   // prefix = the nF-th lowest score; `need` of the pairs with exactly that score are folded: the youngest.
   // Pairs below the threshold are marked at once; pairs on it are collected into a short list first
   // (normally one entry) and ranked among themselves by position.
-  const unsigned thr_key = prefix;
+  thr_key = prefix;
   for (int e = tid; e < nE; e += kUp2Threads) {
     const unsigned k = X.key[e];
     if (k < thr_key) X.pos[e] |= (int)0x80000000;
@@ -210,9 +221,31 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
     }
   }
   __syncthreads();
-  int nGL = 0, nMove = 0;
   for (int w = 0; w < kUp2Threads / 32; ++w) { nGL += X.scan[w][1]; nMove += X.scan[w][2]; }
 
+  }
+  if (PHASE == 1) {
+    // the lists leave through the state's work-list arrays
+    for (int i = tid; i < nF; i += kUp2Threads) g_fold[i] = X.fold_e[i];
+    for (int w = tid; w < nMove; w += kUp2Threads) {
+      g_src[w] = X.mover[w];
+      g_dst[w] = w < nGL ? X.free_slot[w] : cg + (w - nGL);
+    }
+    if (tid == 0) {
+      g_cnt[0] = nF;
+      g_cnt[1] = nMove;
+      L.thr[(size_t)unit * 2 + 0] = __uint_as_float(X.min_keep);
+      L.thr[(size_t)unit * 2 + 1] = __uint_as_float(thr_key);
+    }
+    return;
+  }
+  if (PHASE == 2) {
+    nMove = min(g_cnt[1], kUp2MaxFold);
+    nGL = nMove;                                                     // every destination comes from the list
+    for (int i = tid; i < nF; i += kUp2Threads) X.fold_e[i] = g_fold[i];
+    for (int w = tid; w < nMove; w += kUp2Threads) { X.mover[w] = g_src[w]; X.free_slot[w] = g_dst[w]; }
+    __syncthreads();
+  }
   // ---- 3. gather the folded pairs into the operand tiles (rows >= nF stay zero)
   for (int i = tid; i < nF * nch * 2; i += kUp2Threads) {
     const int row = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
@@ -352,7 +385,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
       scu[dst] = scu[lam + src];
     }
   }
-  if (tid == 0 && ok) {
+  if (PHASE == 0 && tid == 0 && ok) {
     L.thr[(size_t)unit * 2 + 0] = __uint_as_float(X.min_keep);
     L.thr[(size_t)unit * 2 + 1] = __uint_as_float(thr_key);
   }
