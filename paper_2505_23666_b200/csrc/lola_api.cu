@@ -306,6 +306,8 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
     k_select<<<U, 256, sm, s>>>(L, c);
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   }
+  if (st->have_maps && !st->force_chain && (c.mode == UPD_NONE || c.mode == UPD_APPEND) && c.r <= kUp2MaxFold)
+    return launch_apply<DPL>(st, c, s);  // nothing folds: moves from the work lists and the window roll
   LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
   if (c.mode == UPD_SELECT || c.mode == UPD_FOLD_ALL) st->himg_valid = false;   // H changes without its operand image
   k_update<T, DPL><<<U, kUpdThreads, update_smem_floats<DPL>(L.D) * 4, s>>>(L, c);

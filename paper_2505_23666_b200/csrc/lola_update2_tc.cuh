@@ -73,7 +73,10 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lam = L.lam, eta = L.eta;
-  const int cg = c.count_g, nE = cg + c.r, nF = nE - lam;          // 1 <= nF <= min(r, kUp2MaxFold)
+  // PHASE 2 also serves calls that fold nothing (nothing leaves the window yet, or every leaving pair
+  // still finds a free slot): then only the moves and the window roll run
+  const bool fold = c.mode == UPD_SELECT;
+  const int cg = c.count_g, nE = cg + c.r, nF = fold ? nE - lam : 0;   // folding: 1 <= nF <= min(r, kUp2MaxFold)
   float* scu = L.score + (size_t)unit * (lam + L.cmax);
   const uint32_t bar = sbase + kMisc + (uint32_t)offsetof(Update2Misc, bars);
   int* g_fold = L.fold_idx + (size_t)unit * L.cmax;
@@ -84,9 +87,9 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   bool ok = true;
 
   if (tid == 0) { tc::mbar_init(bar, 1); tc::mbar_init_fence(); X.min_keep = 0xffffffffu; X.n_equal = 0; }
-  if (PHASE != 1 && warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
+  if (PHASE != 1 && fold && warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
   // H of the unit streams into shared memory (asynchronous 16-byte copies) meanwhile
-  if (PHASE != 1) {
+  if (PHASE != 1 && fold) {
     const float* Hg = L.H + (size_t)unit * D * d;
     for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
       const int row = i / (d / 4), c4 = i % (d / 4);
@@ -98,7 +101,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   if (PHASE != 2)
     for (int i = tid; i < 4 * 256; i += kUp2Threads) (&X.hist[0][0])[i] = 0;
   // W^T image and zeroed operand tiles
-  if (PHASE != 1) {
+  if (PHASE != 1 && fold) {
     const uint4* img = wt_image + (size_t)h * kblk * 512;
     for (int i = tid; i < kblk * 512; i += kUp2Threads) *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
     for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
@@ -240,12 +243,13 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
     return;
   }
   if (PHASE == 2) {
-    nMove = min(g_cnt[1], kUp2MaxFold);
+    nMove = c.mode == UPD_NONE ? 0 : min(g_cnt[1], kUp2MaxFold);
     nGL = nMove;                                                     // every destination comes from the list
     for (int i = tid; i < nF; i += kUp2Threads) X.fold_e[i] = g_fold[i];
     for (int w = tid; w < nMove; w += kUp2Threads) { X.mover[w] = g_src[w]; X.free_slot[w] = g_dst[w]; }
     __syncthreads();
   }
+  if (fold) {
   // ---- 3. gather the folded pairs into the operand tiles (rows >= nF stay zero)
   for (int i = tid; i < nF * nch * 2; i += kUp2Threads) {
     const int row = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
@@ -371,6 +375,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
     uint4* img4 = reinterpret_cast<uint4*>(ht_image + (size_t)unit * (2 * d * 64));
     for (int i = tid; i < 2 * d * 128 / 16; i += kUp2Threads) img4[i] = *reinterpret_cast<const uint4*>(sm + S::kt + (size_t)i * 16);
   }
+  }  // fold
   // ---- 4. leaving pairs that stay: into the freed slots, then into the slots beyond count_g
   for (int i = tid; i < nMove * nch * 2; i += kUp2Threads) {
     const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
@@ -382,7 +387,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
     *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
     if (rem == 0) {
       L.gpos[(size_t)unit * lam + dst] = c.r_pos0 + src;
-      scu[dst] = scu[lam + src];
+      scu[dst] = fold ? scu[lam + src] : CUDART_NAN_F;               // never scored while the cache still has room
     }
   }
   if (PHASE == 0 && tid == 0 && ok) {
@@ -403,7 +408,7 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   if (!ok && tid == 0) atomicOr(L.status, 32);
   tc::fence_before_sync();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tmem, 256);
+  if (fold && warp == 0) tc::tmem_dealloc(X.tmem_slot, 256);
 }
 
 // Rebuilds the bf16 operand image of H for every unit (after a path that changed H without
