@@ -199,3 +199,22 @@ def test_cfg2_full():
     summ = drive(ls, wl.tokens, wl.chunk)
     print("cfg2", summ)
     assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100)
+
+
+def test_cfg4_needles_full_length():
+    """The long-context workload at full size (131072 tokens, 8 units): outputs of every chunk against the
+    oracle, the memories after every chunk, and the number of planted pairs that end in the sparse cache."""
+    wl = WORKLOADS["cfg4"]
+    ls = Lockstep(wl, threads=8)
+    nch = wl.tokens // wl.chunk
+    for c in range(nch):
+        ls.prefill(c * wl.chunk, wl.chunk)
+    summ = ls.summary()
+    g = ls.layer.read_state()
+    want = set(int(p) for p in ls.inputs.needle_pos)
+    gpu_count = np.array([[sum(int(p) in want for p in g["sparse_pos"][b, h]) for h in range(wl.n_kv_heads)]
+                          for b in range(wl.batch)])
+    orc_count = ls.oracle.needle_count(ls.inputs.needle_pos)
+    print("cfg4", summ, "needles in the sparse cache (oracle / library):", int(orc_count.sum()), int(gpu_count.sum()))
+    assert np.array_equal(gpu_count, orc_count)
+    assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100), summ
