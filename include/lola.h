@@ -13,9 +13,12 @@
  * Conventions for every entry point
  *   - All tensors are row-major with the head dimension innermost and contiguous.
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are ordinary
- *     host memory.  The library never allocates or frees device memory and creates no streams;
- *     the caller owns every buffer (state, W, q, k, v, out) and must keep W and the state buffer
- *     alive for the life of the handle.
+ *     host memory.  The library never allocates or frees device memory; the caller owns every
+ *     buffer (state, W, q, k, v, out) and must keep W and the state buffer alive for the life of
+ *     the handle.  A handle of a bf16 layer holds two host-side objects of its own, a second
+ *     non-blocking stream and a pair of events: lola_prefill_chunk uses them to run the scoring of
+ *     the eligible set beside the attention kernel (both only read the memories) and joins them
+ *     on the caller's stream before anything is written, so the caller sees one ordered stream.
  *   - Work is enqueued on the given stream (a cudaStream_t passed as void*; NULL = legacy default
  *     stream) and the call returns without synchronising unless stated otherwise.  All calls on
  *     one state must be issued on one stream, or be ordered by the caller.
@@ -102,7 +105,8 @@ typedef struct lola_state_view {
 } lola_state_view;
 
 /* Device bytes the caller must provide for one state (a multiple of 256).  0 if cfg is invalid.
- * Holds H, s, the sparse cache with positions and scores, the window ring, and the small per-unit
+ * Holds H, s, the sparse cache with positions and scores, the window ring, for bf16 layers with
+ * feat_half = 64 the tensor-core operand images of W (per KV head) and of H (per unit), and the small per-unit
  * work lists the update kernels pass to each other.                                             */
 size_t lola_state_bytes(const lola_config* cfg);
 
