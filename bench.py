@@ -33,6 +33,29 @@ if ROOT not in sys.path:
 METRIC = "LoLA tokens/s per layer"
 UNIT = "tokens/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch from an ncu capture (profiles/), valid only
+# while the kernel's source is the one that was captured (first 16 hex digits of its SHA-256)
+NCU_TRAFFIC = {
+    "decode": {"source": "paper_2505_23666_b200/csrc/lola_decode_tc.cuh", "sha256_16": "c1075588157eadeb",
+               "bytes_per_launch": 302.6e6, "units": 512},
+}
+
+
+def ncu_traffic(kind, units):
+    """DRAM traffic of one launch of the dominant kernel per the committed ncu capture, scaled by the units a
+    launch processes; None when the kernel has changed since the capture."""
+    import hashlib
+    ent = NCU_TRAFFIC.get(kind)
+    if not ent:
+        return None
+    try:
+        with open(os.path.join(ROOT, ent["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != ent["sha256_16"]:
+                return None
+    except OSError:
+        return None
+    return ent["bytes_per_launch"] * units / ent["units"]
+
 
 # ----------------------------------------------------------------------------- algorithmic work
 def geometry(wl, n_seen, n):
@@ -421,7 +444,8 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
                 "d2h_bytes_per_step": hout.numel() * hout.element_size(), "steps": e2e_steps},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": "+".join(sorted(kms)) + " (all kernels of one decode call)",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": (ncu_traffic("decode", wl.units) if "decode" in kms and len(kms) == 1 else None),
                      "peak_source": peaks["source"], "bytes_per_call": step_bytes, "flops_per_call": step_flops,
                      "launch_us": kernel_ms_per_call * 1e3,
                      "kernel_us_per_call": {k: v / S * 1e3 for k, v in kms.items()}},
