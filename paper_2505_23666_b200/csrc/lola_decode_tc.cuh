@@ -72,7 +72,7 @@ struct DecodeMisc {
   float cand_z[kDecMaxTiles][kDecQ];
   uint4 cand_v[kDecMaxTiles][16];    // value row, bf16
   uint4 cand_phi[kDecMaxTiles][16];  // feature row, bf16
-  uint64_t bars[8];
+  uint64_t bars[12];
   uint32_t tmem_slot;
 };
 static_assert(sizeof(DecodeMisc) <= 28672, "misc region too small");
@@ -153,32 +153,29 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   bool ok = true;
 
   if (tid == 0) {
-    for (int i = 0; i < 8; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + 8u * i, 1);
+    for (int i = 0; i < 10; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + 8u * i, 1);
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
   __syncthreads();
   // first tile of each row group starts to stream while the operands below are prepared
-  if (lead && wg < NT) {
-    decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, wg, nGB, nRB, unit, bar_k);
-    decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, wg, nGB, nRB, unit, bar_v);
+  // H (fp32, 64 KB at d = 128) comes in by two bulk copies into the two value buffers, which the first
+  // value tiles only need later; W^T by bulk copies straight into the operand rows
+  const uint32_t bar_h = sbase + S::misc + (uint32_t)offsetof(DecodeMisc, bars) + 64u;
+  const uint32_t bar_w = bar_h + 8u;
+  if (tid == 0) {
+    const float* Hg = L.H + (size_t)unit * D * d;
+    tc::mbar_expect_tx(bar_h, (uint32_t)(D * d * 4));
+    tc::bulk_copy_g2s(sbase + S::stage0 + S::st_v, Hg, 64u * d * 4u, bar_h);
+    tc::bulk_copy_g2s(sbase + S::stage0 + S::stage_bytes + S::st_v, Hg + 64 * d, 64u * d * 4u, bar_h);
+    tc::mbar_expect_tx(bar_w, (uint32_t)kblk * 8192u);
+    for (int kb = 0; kb < kblk; ++kb)
+      tc::bulk_copy_g2s(sbase + S::b1 + (uint32_t)kb * S::b1_blk, wt_image + ((size_t)h * kblk + kb) * 512, 8192u, bar_w);
   }
+  if (lead && wg < NT) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, wg, nGB, nRB, unit, bar_k);
 
   // ---- operands that stay for the whole unit
-  constexpr int HI = d * (D / 8) / kDecThreads;
-  float hreg[HI][8];
-  const float* Hg = L.H + (size_t)unit * D * d;
   {
-    // H (fp32 [D][d]) -> bf16 H^T, K-major: row c, 64 j per 128-byte row, two j blocks.  A thread
-    // gathers 8 consecutive j of one column c (each load coalesced over the warp's 32 columns).  All
-    // loads are issued here; they are converted and stored after the small query-side work below.
-#pragma unroll
-    for (int it = 0; it < HI; ++it) {
-      const int i = tid + it * kDecThreads;
-      const int cc = i % d, jc = i / d;
-#pragma unroll
-      for (int jj = 0; jj < 8; ++jj) hreg[it][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
-    }
     // rows d, d+1: s as the sum of two bf16 parts (phi . s_hi + phi . s_lo keeps the fp32 normaliser)
     if (tid < D) {
       const float sv = L.s[(size_t)unit * D + tid];
@@ -193,10 +190,6 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
       *reinterpret_cast<uint4*>(sm + S::ht + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
     }
-    // W^T image (prepared once per layer in the operand layout): rows 0..63 of each K block of B1
-    const uint4* img = wt_image + (size_t)h * kblk * 512;
-    for (int i = tid; i < kblk * 512; i += kDecThreads)
-      *reinterpret_cast<uint4*>(sm + S::b1 + (i >> 9) * S::b1_blk + (i & 511) * 16) = img[i];
     // query rows: B1 rows 64..79 (rows >= g are zero) and an fp32 copy
     constexpr int per_row = d / 8;
     for (int i = tid; i < 16 * per_row; i += kDecThreads) {
@@ -226,6 +219,7 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       *reinterpret_cast<uint4*>(sm + S::stage0 + S::stage_bytes + S::st_pt + i * 16) = make_uint4(0, 0, 0, 0);
     }
   }
+  ok = tc::mbar_wait(bar_w, 0) && ok;
   __syncthreads();
   // u = q W on the CUDA cores (g rows only) from the W^T operand image
   for (int i = tid; i < g * F; i += kDecThreads) {
@@ -274,16 +268,23 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     zz = warp_sum(zz);
     if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * sl2; }
   }
-#pragma unroll
-  for (int it = 0; it < HI; ++it) {
-    const int i = tid + it * kDecThreads;
+  // H (fp32 [D][d], staged in the value buffers) -> bf16 H^T, K-major: row c, 64 j per 128-byte row, two
+  // j blocks.  A thread gathers 8 consecutive j of one column c (lanes = consecutive columns: no conflicts).
+  ok = tc::mbar_wait(bar_h, 0) && ok;
+  for (int i = tid; i < d * (D / 8); i += kDecThreads) {
     const int cc = i % d, jc = i / d;
-    *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(hreg[it]);
+    const float* src = reinterpret_cast<const float*>(sm + S::stage0 + (jc >> 3) * S::stage_bytes + S::st_v) + ((jc & 7) * 8) * d + cc;
+    float f8[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) f8[jj] = src[jj * d];
+    *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
   }
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
+  // the value buffers are free now: the first value tiles start to stream
+  if (lead && wg < NT) decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, wg, nGB, nRB, unit, bar_v);
   const uint32_t tmem = X.tmem_slot;
   const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
   const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // [U | Z], then [P | den]
