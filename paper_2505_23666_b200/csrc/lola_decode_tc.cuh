@@ -405,6 +405,39 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     for (int r = 0; r < QR; ++r)
       m_new[r] = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[wg][0][r], X.redmax[wg][1][r])),
                        fmaxf(X.redmax[wg][2][r], X.redmax[wg][3][r]));
+    // ---- softmax weights of the tile (bf16; the sums use the rounded weights): this thread's query rows.
+    // Computed while the second product runs, for every valid row; the row that turns out to have the
+    // tile's lowest score takes its weights back below.
+    float pw[QR];
+    {
+      bool moved = false;
+      float alpha[QR];
+#pragma unroll
+      for (int r = 0; r < QR; ++r) {
+        alpha[r] = tc::fast_exp2(m_run[r] - m_new[r]);
+        moved = moved || (m_new[r] != m_run[r]);
+        lpart[r] *= alpha[r];
+        m_run[r] = m_new[r];
+        pw[r] = 0.f;
+      }
+#pragma unroll
+      for (int r = 0; r < QR; ++r) {          // static indices keep z, m_new, lpart in registers
+        if ((r / (QR / 2)) == hf) {
+          const float p = valid ? tc::fast_exp2(z[r] - m_new[r]) : 0.f;
+          const uint32_t pb = pack_bf16x2(p, 0.f);
+          pw[r] = bf16lo_f(pb);
+          lpart[r] += pw[r];
+          *reinterpret_cast<unsigned short*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = (unsigned short)pb;
+        }
+      }
+      if (have_o && moved && hf == 0) {          // `moved` is uniform over the row group
+        float ov[8];
+        tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+        for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
+        tc::tmem_st8(tm_o + lane_addr, ov);
+      }
+    }
 
     ok = tc::mbar_wait(bar_v, pv) && ok; pv ^= 1;
     ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
@@ -493,32 +526,14 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
         for (int i = 0; i < 32; ++i) dst[i] = pr[i];
       }
     }
-    // ---- softmax weights of the tile (bf16; the sums use the rounded weights): query rows 4 hf .. 4 hf + 3
-    {
-      bool moved = false;
-      float alpha[QR];
+    // the row left out of O^T: take its weights back (they were written before the scores were known)
+    if (left_out) {
 #pragma unroll
       for (int r = 0; r < QR; ++r) {
-        alpha[r] = tc::fast_exp2(m_run[r] - m_new[r]);
-        moved = moved || (m_new[r] != m_run[r]);
-        lpart[r] *= alpha[r];
-        m_run[r] = m_new[r];
-      }
-#pragma unroll
-      for (int r = 0; r < QR; ++r) {          // static indices keep z, m_new, lpart in registers
         if ((r / (QR / 2)) == hf) {
-          float p = (valid && !left_out) ? tc::fast_exp2(z[r] - m_new[r]) : 0.f;
-          const uint32_t pb = pack_bf16x2(p, 0.f);
-          lpart[r] += bf16lo_f(pb);
-          *reinterpret_cast<unsigned short*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = (unsigned short)pb;
+          lpart[r] -= pw[r];
+          *reinterpret_cast<unsigned short*>(stage_p + S::st_pt + (t >> 6) * 2048 + tc::sw128_off(r, (t & 63) >> 3) + (t & 7) * 2) = 0;
         }
-      }
-      if (have_o && moved && hf == 0) {          // `moved` is uniform over the row group
-        float ov[8];
-        tc::tmem_ld8(tm_o + lane_addr, ov);
-#pragma unroll
-        for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
-        tc::tmem_st8(tm_o + lane_addr, ov);
       }
     }
     tc::fence_async_smem();
@@ -533,8 +548,11 @@ k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
                         tc::make_desc_sw128(stage + S::st_pt + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc3,
                         (have_o || ks > 0) ? 1u : 0u);
       tc::mma_commit(bar_mma3);
-      // the value buffer is free once this product is done; everybody else meets the leader again at
-      // the next barrier, before anything of this product's operands or O^T is touched
+    }
+    if ((tid & 255) == 32) {
+      // a second thread waits for this product (the leader goes on to issue the next tile's first one):
+      // the value buffer is free once it is done; everybody else meets this thread again at the next
+      // barrier, before anything of this product's operands or O^T is touched
       ok = tc::mbar_wait(bar_mma3, pm3) && ok;
       tc::fence_after_sync();
       if (tile + 2 < NT) decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_v);
