@@ -249,6 +249,34 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
     for (int w = tid; w < nMove; w += kUp2Threads) { X.mover[w] = g_src[w]; X.free_slot[w] = g_dst[w]; }
     __syncthreads();
   }
+  // ---- leaving pairs that stay: into the freed slots, then into the slots beyond count_g
+  auto do_movers = [&](int t0, int nt) {
+    for (int i = t0; i < nMove * nch * 2; i += nt) {
+      const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+      const int src = X.mover[w];
+      const int dst = w < nGL ? X.free_slot[w] : cg + (w - nGL);
+      const T *kp, *vp;
+      locate_leaving<T>(L, c, unit, b, h, c.r_pos0 + src, kp, vp);
+      T* dp = (isv ? (T*)L.gv : (T*)L.gk) + ((size_t)unit * lam + dst) * d;
+      *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
+      if (rem == 0) {
+        L.gpos[(size_t)unit * lam + dst] = c.r_pos0 + src;
+        scu[dst] = fold ? scu[lam + src] : CUDART_NAN_F;             // never scored while the cache still has room
+      }
+    }
+  };
+  // ---- the window takes the chunk's last eta tokens (after every read of the rows it replaces)
+  auto do_roll = [&](int t0, int nt) {
+    if (eta <= 0) return;
+    const int first = max(0, c.n - eta);
+    for (int i = t0; i < (c.n - first) * nch * 2; i += nt) {
+      const int ci = first + i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+      const int p = c.n_seen + ci;
+      const T* sp = (isv ? (const T*)c.v : (const T*)c.k) + (((size_t)b * c.n + ci) * L.Hkv + h) * d;
+      T* dp = (isv ? (T*)L.wv : (T*)L.wk) + ((size_t)unit * eta + (p % eta)) * d;
+      *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>(sp + ch * 8);
+    }
+  };
   if (fold) {
   // ---- 3. gather the folded pairs into the operand tiles (rows >= nF stay zero)
   for (int i = tid; i < nF * nch * 2; i += kUp2Threads) {
@@ -278,7 +306,10 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
                       tc::make_idesc_bf16(128, 64, false, false), ks > 0);
     tc::mma_commit(bar);
   }
-  ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1;
+  // the upper half of the block moves the staying pairs meanwhile (the gather above has read every
+  // slot and ring row the fold needs; the movers only read ring rows and write freed or new slots)
+  if (tid >= 256) do_movers(tid - 256, kUp2Threads - 256);
+  else { ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1; }
   tc::fence_after_sync();
   if (tid < 256) {                                                   // one thread pair per row: half of the feature map each
     float e[64];
@@ -332,7 +363,8 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
                       tc::make_idesc_bf16(128, d + 16, true, true), ks > 0);
     tc::mma_commit(bar);
   }
-  ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1;
+  if (tid >= 256) do_roll(tid - 256, kUp2Threads - 256);             // the movers' reads of the ring ended at the barrier above
+  else { ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1; }
   tc::fence_after_sync();
   if (tid < 256 && ok) {                                             // row j = t, columns [hf * d/2, +d/2)
     // H += dH in the shared-memory copy (this thread owns the half row) and the same values as bf16 in
@@ -376,34 +408,14 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
     for (int i = tid; i < 2 * d * 128 / 16; i += kUp2Threads) img4[i] = *reinterpret_cast<const uint4*>(sm + S::kt + (size_t)i * 16);
   }
   }  // fold
-  // ---- 4. leaving pairs that stay: into the freed slots, then into the slots beyond count_g
-  for (int i = tid; i < nMove * nch * 2; i += kUp2Threads) {
-    const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
-    const int src = X.mover[w];
-    const int dst = w < nGL ? X.free_slot[w] : cg + (w - nGL);
-    const T *kp, *vp;
-    locate_leaving<T>(L, c, unit, b, h, c.r_pos0 + src, kp, vp);
-    T* dp = (isv ? (T*)L.gv : (T*)L.gk) + ((size_t)unit * lam + dst) * d;
-    *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
-    if (rem == 0) {
-      L.gpos[(size_t)unit * lam + dst] = c.r_pos0 + src;
-      scu[dst] = fold ? scu[lam + src] : CUDART_NAN_F;               // never scored while the cache still has room
-    }
+  if (!fold) {
+    do_movers(tid, kUp2Threads);
+    __syncthreads();                                                 // ring rows are read above before they are replaced
+    do_roll(tid, kUp2Threads);
   }
   if (PHASE == 0 && tid == 0 && ok) {
     L.thr[(size_t)unit * 2 + 0] = __uint_as_float(X.min_keep);
     L.thr[(size_t)unit * 2 + 1] = __uint_as_float(thr_key);
-  }
-  __syncthreads();                                                   // ring rows are read above before they are replaced
-  if (eta > 0) {
-    const int first = max(0, c.n - eta);
-    for (int i = tid; i < (c.n - first) * nch * 2; i += kUp2Threads) {
-      const int ci = first + i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
-      const int p = c.n_seen + ci;
-      const T* sp = (isv ? (const T*)c.v : (const T*)c.k) + (((size_t)b * c.n + ci) * L.Hkv + h) * d;
-      T* dp = (isv ? (T*)L.wv : (T*)L.wk) + ((size_t)unit * eta + (p % eta)) * d;
-      *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>(sp + ch * 8);
-    }
   }
   if (!ok && tid == 0) atomicOr(L.status, 32);
   tc::fence_before_sync();
