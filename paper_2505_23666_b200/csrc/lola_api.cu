@@ -16,6 +16,7 @@
 #include "lola_score_tc.cuh"
 #include "lola_attend_tc.cuh"
 #include "lola_decode_tc.cuh"
+#include "lola_decode2_tc.cuh"
 #include "lola_score2_tc.cuh"
 #include "lola_update2_tc.cuh"
 #include "lola_attend2_tc.cuh"
@@ -343,6 +344,15 @@ template <int DPL>
 int launch_decode_fused(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   LaunchScope scope(st, LOLA_KERNEL_DECODE, s);
+  const int n_tiles = (L.lam / 64 + (L.eta + 63) / 64 + 1) / 2;
+  const uint4* wt = (const uint4*)(st->base + st->lay.wt);
+  if (n_tiles <= kDec2MaxTiles) {          // the pipelined kernel; longer units run the two-row-group kernel
+    if (L.g <= 4)
+      k_decode2_tc<DPL, 4><<<L.B * L.Hkv, kDec2Threads, DecodeSmem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, wt);
+    else
+      k_decode2_tc<DPL, 8><<<L.B * L.Hkv, kDec2Threads, DecodeSmem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, wt);
+    return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+  }
   if (L.g <= 4)
     k_decode_tc<DPL, 4><<<L.B * L.Hkv, kDecThreads, DecodeSmem<DPL>::bytes, s>>>(
         L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, (const uint4*)(st->base + st->lay.wt));
@@ -447,14 +457,18 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       e[2] = cudaFuncSetAttribute(k_score2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<4>::bytes);
       e[3] = cudaFuncSetAttribute(k_update2_tc<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<4>::bytes);
       e[4] = cudaFuncSetAttribute(k_attend2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<4>::bytes);
+      e[5] = cudaFuncSetAttribute(k_decode2_tc<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
+      e[6] = cudaFuncSetAttribute(k_decode2_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
     } else {
       e[0] = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[1] = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[2] = cudaFuncSetAttribute(k_score2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Score2Smem<2>::bytes);
       e[3] = cudaFuncSetAttribute(k_update2_tc<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Update2Smem<2>::bytes);
       e[4] = cudaFuncSetAttribute(k_attend2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<2>::bytes);
+      e[5] = cudaFuncSetAttribute(k_decode2_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
+      e[6] = cudaFuncSetAttribute(k_decode2_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
     }
-    for (int i = 0; i < 5; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
+    for (int i = 0; i < 7; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
   }
   if (rc == LOLA_OK && st->have_maps) {
     // host-side objects only (no device memory): a second stream and two events to run the scoring

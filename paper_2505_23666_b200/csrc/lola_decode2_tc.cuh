@@ -1,0 +1,708 @@
+// The generation step (Eq. 11-14) as ONE kernel, organised as a pipeline of roles (the steady state of
+// a bf16 layer with F = 64, caches full, one pair leaving the window; at most 8 row tiles per unit).
+// Same arithmetic and the same per-tile products as k_decode_tc; what differs is who does what:
+//
+//   feature group (warps 0-7)   per tile: q.k columns and their row maxima, softmax weights (bf16) into
+//                               the Pr^T operand, the feature map of U into tensor memory
+//   score group   (warps 8-15)  per tile: Eq. 10 from [P | den] and the value tile, the tile's lowest
+//                               score, the row left out of O^T, the running sums of the weights
+//   warp 16, one thread         issues [U | Z] = K [W | Q^T] and [P | den] = phi [H | s]; key-tile loads
+//   warp 17, one thread         issues O^T += V^T Pr^T; value-tile loads
+//
+// The two groups work on different tiles at the same time: [U | Z] and phi are double-buffered in
+// tensor memory, so while the score group is busy with tile t the feature group already works on
+// tile t + 1 and the tensor core on the products between them.  Every hand-over is an mbarrier; every
+// wait is bounded, and a wait that runs out raises the block's abort word (bit 8 of the status word).
+#pragma once
+#include "lola_decode_tc.cuh"
+
+namespace lola {
+
+constexpr int kDec2MaxTiles = 8;
+constexpr int kDec2Threads = 576;      // 16 compute warps + 2 issuing warps
+
+struct Decode2Misc {
+  float qf[kDecQ][128];          // query rows, fp32
+  float phiq_f[kDecQ][128];      // phi(q) rounded to bf16, as fp32
+  float u_s[kDecQ][64];
+  float knew[128], vnew[128];
+  float zn[kDecQ], lden[kDecQ], dotL[kDecQ];
+  float redmax[2][4][kDecQ];
+  float m_s[2][kDecQ];           // running maximum after tile t (log2 units)
+  float z_s[2][kDecQ][128];      // q.k of the tile's rows (log2 units)
+  unsigned long long redkey[4];
+  float red12[4][2];
+  float ssp[128];                // partial squared errors of the second half of the value columns
+  float l_s[4][kDecQ];
+  int moved[2][2];               // a running maximum grew in tile t (per half of the query rows)
+  unsigned long long cand_key[kDec2MaxTiles];
+  float cand_score[kDec2MaxTiles], cand_min2[kDec2MaxTiles];
+  int cand_row[kDec2MaxTiles];
+  float cand_z[kDec2MaxTiles][kDecQ];
+  uint4 cand_v[kDec2MaxTiles][16];    // value row, bf16
+  uint4 cand_phi[kDec2MaxTiles][16];  // feature row, bf16
+  uint64_t bars[20];
+  uint32_t tmem_slot;
+  int abort_word;
+};
+static_assert(sizeof(Decode2Misc) <= 28672, "misc region too small");
+
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}\n"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
+template <int DPL, int QR>
+__global__ void __launch_bounds__(kDec2Threads, 1)
+k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
+             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image) {
+  using S = DecodeSmem<DPL>;
+  constexpr int d = DPL * 32;
+  constexpr int kblk = d / 64;
+  constexpr int F = 64, D = 128;
+  constexpr int HC = d / 2;                  // value columns per thread of a row pair
+  constexpr int QH = QR / 2;                 // query rows per thread of a row pair
+  constexpr float kLog2e = 1.4426950408889634f;
+  typedef __nv_bfloat16 T;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = tc::smem_u32(sm);
+  Decode2Misc& X = *reinterpret_cast<Decode2Misc*>(sm + S::misc);
+
+  const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int role = warp < 8 ? 0 : (warp < 16 ? 1 : warp - 14);   // 0 feature, 1 score, 2 / 3 issuing threads
+  const int gtid = tid & 255;                // index inside a compute group
+  const int gw = warp & 7;
+  const int wq = gw & 3;                     // tensor-memory lane quadrant of this warp (= warp % 4)
+  const int hf = gw >> 2;                    // which half of the row's work this thread does
+  const int t = wq * 32 + lane;              // row of the tile = tensor-memory lane
+  const int lam = L.lam, eta = L.eta, g = L.g;
+  const int nGB = lam / 64, nRB = (eta + 63) / 64, NT = (nGB + nRB + 1) / 2;
+  const int s_ev = c.n_seen % eta;           // ring slot of the pair that leaves = slot the new pair takes
+  const int pos_ev = c.n_seen - eta;
+  const float sl2 = L.scale * kLog2e;        // q.k in log2 units
+  float* scu = L.score + (size_t)unit * (lam + L.cmax);
+  volatile int* abw = &X.abort_word;
+
+  const uint32_t bars = sbase + S::misc + (uint32_t)offsetof(Decode2Misc, bars);
+  auto bar_kfull = [&](int i) { return bars + 8u * (uint32_t)i; };
+  auto bar_vfull = [&](int i) { return bars + 16u + 8u * (uint32_t)i; };
+  auto bar_u = [&](int i) { return bars + 32u + 8u * (uint32_t)i; };
+  auto bar_phidone = [&](int i) { return bars + 48u + 8u * (uint32_t)i; };
+  const uint32_t bar_p = bars + 64u, bar_pfree = bars + 72u;
+  auto bar_ptready = [&](int i) { return bars + 80u + 8u * (uint32_t)i; };
+  auto bar_o = [&](int i) { return bars + 96u + 8u * (uint32_t)i; };
+  const uint32_t bar_w = bars + 112u, bar_h = bars + 120u, bar_ht = bars + 128u;
+  auto stage_k = [&](int i) { return sbase + S::stage0 + (uint32_t)i * S::stage_bytes + S::st_k; };
+  auto stage_v = [&](int i) { return sbase + S::stage0 + (uint32_t)i * S::stage_bytes + S::st_v; };
+  auto stage_pt = [&](int i) { return S::stage0 + (uint32_t)i * S::stage_bytes + S::st_pt; };   // offset from sm
+
+  if (tid == 0) {
+    X.abort_word = 0;
+    for (int i = 0; i < 17; ++i) {
+      const bool group = (i == 6 || i == 7 || i == 9 || i == 10 || i == 11 || i == 16);
+      tc::mbar_init(bars + 8u * i, group ? 256u : 1u);
+    }
+    tc::mbar_init_fence();
+  }
+  if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
+  __syncthreads();
+  if (tid == 17 * 32) {
+    // W^T straight into the operand rows; H (fp32) into the key and value buffers of stage 1, which
+    // the second tile only needs later; the first tile starts to stream at once
+    tc::mbar_expect_tx(bar_w, (uint32_t)kblk * 8192u);
+    for (int kb = 0; kb < kblk; ++kb)
+      tc::bulk_copy_g2s(sbase + S::b1 + (uint32_t)kb * S::b1_blk, wt_image + ((size_t)h * kblk + kb) * 512, 8192u, bar_w);
+    decode_issue_tile<DPL>(stage_k(0), &tm_gk, &tm_wk, 0, nGB, nRB, unit, bar_kfull(0));
+    const float* Hg = L.H + (size_t)unit * D * d;
+    tc::mbar_expect_tx(bar_h, (uint32_t)(D * d * 4));
+    tc::bulk_copy_g2s(stage_k(1), Hg, 64u * d * 4u, bar_h);
+    tc::bulk_copy_g2s(stage_v(1), Hg + 64 * d, 64u * d * 4u, bar_h);
+    decode_issue_tile<DPL>(stage_v(0), &tm_gv, &tm_wv, 0, nGB, nRB, unit, bar_vfull(0));
+  }
+
+  // ---- operands that stay for the whole unit (compute warps)
+  if (role < 2) {
+    // rows d, d+1: s as the sum of two bf16 parts (phi . s_hi + phi . s_lo keeps the fp32 normaliser)
+    if (tid < D) {
+      const float sv = L.s[(size_t)unit * D + tid];
+      const __nv_bfloat16 hi = __float2bfloat16_rn(sv);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(sv - __bfloat162float(hi));
+      const int ch = (tid & 63) >> 3;
+      *reinterpret_cast<T*>(sm + S::ht + (tid >> 6) * S::ht_blk + tc::sw128_off(d, ch) + (tid & 7) * 2) = hi;
+      *reinterpret_cast<T*>(sm + S::ht + (tid >> 6) * S::ht_blk + tc::sw128_off(d + 1, ch) + (tid & 7) * 2) = lo;
+    }
+    // rows d+2 .. d+15 of both j blocks: zero
+    for (int i = tid; i < 2 * 14 * 8; i += 512) {
+      const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
+      *reinterpret_cast<uint4*>(sm + S::ht + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
+    }
+    // query rows: B1 rows 64..79 (rows >= g are zero) and an fp32 copy
+    constexpr int per_row = d / 8;
+    for (int i = tid; i < 16 * per_row; i += 512) {
+      const int r = i / per_row, ch = i % per_row;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (r < g) val = *reinterpret_cast<const uint4*>((const T*)c.q + ((size_t)b * L.Hq + h * g + r) * d + ch * 8);
+      *reinterpret_cast<uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(64 + r, ch & 7)) = val;
+      if (r < QR) {
+        const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&val);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float2 ff = __bfloat1622float2(v2[q]);
+          X.qf[r][ch * 8 + 2 * q] = ff.x;
+          X.qf[r][ch * 8 + 2 * q + 1] = ff.y;
+        }
+      }
+    }
+    if (tid < d) {
+      X.knew[tid] = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + tid);
+      X.vnew[tid] = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + tid);
+    }
+    if (tid < kDec2MaxTiles) { X.cand_key[tid] = ~0ull; X.cand_score[tid] = CUDART_INF_F; X.cand_min2[tid] = CUDART_INF_F; X.cand_row[tid] = 0; }
+    // zero phi(Q) and both Pr^T tiles
+    for (int i = tid; i < 256; i += 512) {
+      *reinterpret_cast<uint4*>(sm + S::phiq + i * 16) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(sm + stage_pt(0) + i * 16) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(sm + stage_pt(1) + i * 16) = make_uint4(0, 0, 0, 0);
+    }
+    tc::fence_async_smem();
+  }
+  __syncthreads();
+
+  const uint32_t tmem = X.tmem_slot;
+  const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+  auto tm_uz = [&](int i) { return tmem + (uint32_t)i * 96u; };          // [U | Z]: 80 columns, two buffers
+  const uint32_t tm_o = tmem + 176u;                                       // O^T: lanes = value column, 16 columns = query rows
+  auto tm_phi = [&](int i) { return tmem + 192u + (uint32_t)i * 64u; };   // phi tile, bf16 pairs: 64 columns, two buffers
+  const uint32_t tm_p = tmem + 320u;                                       // [P | den]: d + 16 columns
+  const uint32_t idesc1 = tc::make_idesc_bf16(128, 80, false, false);
+  const uint32_t idesc2 = tc::make_idesc_bf16(128, d + 16, false, false);
+  const uint32_t idesc0 = tc::make_idesc_bf16(128, 16, false, false);
+  const uint32_t idesc3 = tc::make_idesc_bf16(128, 16, true, false);
+  bool ok = true;
+
+  if (role == 2) {
+    // =================== products of the feature side, key tiles ===================
+    if (lane == 0) {
+      // operand descriptors: the address field (units of 16 bytes) takes the offset of a K step
+      const uint64_t dk0 = tc::make_desc_sw128(stage_k(0), 16, 1024), dk1 = tc::make_desc_sw128(stage_k(1), 16, 1024);
+      const uint64_t db1 = tc::make_desc_sw128(sbase + S::b1, 16, 1024), dht = tc::make_desc_sw128(sbase + S::ht, 16, 1024);
+      auto issue_mma1 = [&](int tile) {
+        const uint64_t dk = (tile & 1) ? dk1 : dk0;
+        const uint32_t tmu = tm_uz(tile & 1);
+#pragma unroll
+        for (int ks = 0; ks < d / 16; ++ks)
+          tc::mma_bf16_ss(tmu, dk + (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                          db1 + (uint64_t)(((ks >> 2) * S::b1_blk + (ks & 3) * 32) >> 4), idesc1, ks > 0);
+        tc::mma_commit(bar_u(tile & 1));
+      };
+      // key tiles: tile x + 2 streams into the buffer of tile x once that tile's first product is complete
+      int next_k = 2;                                  // tiles 0 and 1 are loaded by the prologue
+      int n1 = 0;                                      // first products issued so far
+      auto load_k = [&]() {
+        decode_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
+        ++next_k;
+      };
+      auto poll_k = [&]() {
+        while (next_k < NT && next_k - 2 < n1 && mbar_test(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u)) load_k();
+      };
+      // waits for a barrier and keeps the key stream going meanwhile
+      auto wait_poll = [&](uint32_t bar, uint32_t parity) {
+        for (uint32_t it = 0; it < 64u; ++it) {
+          uint32_t done;
+          asm volatile(
+              "{\n\t"
+              ".reg .pred p;\n\t"
+              "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+              "selp.u32 %0, 1, 0, p;\n\t"
+              "}\n"
+              : "=r"(done)
+              : "r"(bar), "r"(parity)
+              : "memory");
+          if (done) return true;
+          poll_k();
+        }
+        return tc::mbar_wait(bar, parity, abw);
+      };
+      auto mma1 = [&](int tile) {                      // needs: key tile landed, [U | Z] buffer free
+        while (next_k <= tile) {                       // (its load must have been issued)
+          ok = tc::mbar_wait(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u, abw) && ok;
+          load_k();
+        }
+        ok = wait_poll(bar_kfull(tile & 1), (uint32_t)(tile >> 1) & 1u) && ok;
+        tc::fence_after_sync();
+        issue_mma1(tile);
+        ++n1;
+      };
+      ok = tc::mbar_wait(bar_w, 0, abw) && ok;
+      mma1(0);
+      for (int tile = 0; tile < NT; ++tile) {
+        const int i = tile & 1;
+        ok = wait_poll(bar_phidone(i), (uint32_t)(tile >> 1) & 1u) && ok;   // phi(tile) written, [U | Z] of this tile read
+        tc::fence_after_sync();
+        if (tile == 0) {
+          // H^T is in place: stage 1 is free for the second tile; O^T starts as the linear term
+          // H^T phi(Q)^T, with weight exp(0 - m), m = 0 so far
+          ok = tc::mbar_wait(bar_ht, 0, abw) && ok;
+          tc::fence_after_sync();
+          if (NT > 1) {
+            decode_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
+            decode_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
+          }
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
+                            tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc0, ks > 0);
+          tc::mma_commit(bar_o(0));
+        } else {
+          ok = wait_poll(bar_pfree, (uint32_t)(tile - 1) & 1u) && ok;   // [P | den] of the tile before is read
+          tc::fence_after_sync();
+        }
+        const uint32_t tph = tm_phi(i);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ts(tm_p, tph + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
+        tc::mma_commit(bar_p);
+        // first products run two tiles ahead of the feature group: the buffer this tile used is free
+        if (tile == 0 && NT > 1) mma1(1);
+        if (tile + 2 < NT) mma1(tile + 2);
+      }
+    }
+    __syncwarp();
+  } else if (role == 3) {
+    // =================== O^T products, value tiles ===================
+    if (lane == 0) {
+      const uint64_t dv0 = tc::make_desc_sw128(stage_v(0), 16384, 1024), dv1 = tc::make_desc_sw128(stage_v(1), 16384, 1024);
+      const uint64_t dp0 = tc::make_desc_sw128(sbase + stage_pt(0), 16, 1024), dp1 = tc::make_desc_sw128(sbase + stage_pt(1), 16, 1024);
+      for (int tile = 0; tile < NT; ++tile) {
+        const int i = tile & 1;
+        ok = tc::mbar_wait(bar_ptready(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+        tc::fence_after_sync();
+        const uint64_t dv = i ? dv1 : dv0, dp = i ? dp1 : dp0;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          tc::mma_bf16_ss(tm_o, dv + (uint64_t)((ks * 2048) >> 4), dp + (uint64_t)(((ks >> 2) * 2048 + (ks & 3) * 32) >> 4), idesc3, 1u);
+        const int ev = tile + 1;                                      // completion event of this product
+        tc::mma_commit(bar_o(ev & 1));
+        ok = tc::mbar_wait(bar_o(ev & 1), (uint32_t)(ev >> 1) & 1u, abw) && ok;
+        if (tile + 2 < NT) decode_issue_tile<DPL>(stage_v(i), &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_vfull(i));
+      }
+    }
+    __syncwarp();
+  } else if (role == 0) {
+    // =================== feature group ===================
+    // this thread's query rows: [hf * QH, hf * QH + QH)
+    float m_run[QH];
+#pragma unroll
+    for (int r = 0; r < QH; ++r) m_run[r] = 0.f;
+    const bool exp_kind = L.phi_kind == 1;
+    for (int tile = 0; tile < NT; ++tile) {
+      const int i = tile & 1;
+      const int R = tile * 128 + t;
+      const bool valid = R < lam || R - lam < eta;
+      ok = tc::mbar_wait(bar_u(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+      tc::fence_after_sync();
+      float z[QH];
+      {
+        float zraw[QH];
+        if (QH == 4) tc::tmem_ld4(tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<float(&)[4]>(zraw));
+        else tc::tmem_ld2(tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<float(&)[2]>(zraw));
+#pragma unroll
+        for (int r = 0; r < QH; ++r) {
+          z[r] = valid ? zraw[r] * sl2 : -CUDART_INF_F;
+          float wm = warp_max_redux(z[r]);
+          if (lane == 0) X.redmax[i][wq][hf * QH + r] = wm;
+        }
+      }
+      // this thread's half of the feature map: hf = 0: softmax(u), hf = 1: softmax(-u)
+      uint32_t pk2[32];
+      {
+        uint32_t u[64];
+        tc::tmem_ld64u(tm_uz(i) + lane_addr, u);
+        if (hf) tc::phi_half_packed<true>(u, exp_kind, pk2);
+        else tc::phi_half_packed<false>(u, exp_kind, pk2);
+      }
+      if (tile >= 2) {
+        // the buffers of tile - 2: its feature rows and q.k columns were used by the score group, its
+        // Pr^T operand by the O^T product
+        ok = tc::mbar_wait(bar_ptready(i), (uint32_t)((tile - 2) >> 1) & 1u, abw) && ok;
+        const int ev = tile - 1;
+        ok = tc::mbar_wait(bar_o(ev & 1), (uint32_t)(ev >> 1) & 1u, abw) && ok;
+        tc::fence_after_sync();
+      }
+      // bf16 pairs into tensor memory: the A operand of the second product (K index = feature j)
+      tc::tmem_st32u(tm_phi(i) + lane_addr + hf * 32, pk2);
+      tc::named_bar_sync(1, 256);
+      // running maximum of q.k per query row (every valid row counts, also the one that will be folded:
+      // any m >= the true maximum leaves Eq. 14 unchanged), then the softmax weights of the tile (bf16;
+      // the sums use the rounded weights)
+      uint8_t* ptile = sm + stage_pt(i);
+      bool moved = false;
+#pragma unroll
+      for (int r = 0; r < QH; ++r) {
+        const int rr = hf * QH + r;
+        const float m_new = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[i][0][rr], X.redmax[i][1][rr])),
+                                  fmaxf(X.redmax[i][2][rr], X.redmax[i][3][rr]));
+        moved = moved || (m_new != m_run[r]);
+        m_run[r] = m_new;
+        const float p = valid ? tc::fast_exp2(z[r] - m_new) : 0.f;
+        *reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2) =
+            (unsigned short)pack_bf16x2(p, 0.f);
+        X.z_s[i][rr][t] = z[r];
+      }
+      if ((gtid & 127) == 0) {
+#pragma unroll
+        for (int r = 0; r < QH; ++r) X.m_s[i][hf * QH + r] = m_run[r];
+        X.moved[i][hf] = moved ? 1 : 0;
+      }
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      tc::mbar_arrive(bar_phidone(i));
+    }
+  } else {
+    // =================== score group ===================
+    // first: what the linear term needs.  u = q W on the CUDA cores (g rows only) from the W^T operand image
+    ok = tc::mbar_wait(bar_w, 0, abw) && ok;
+    for (int i = gtid; i < g * F; i += 256) {
+      const int r = i >> 6, f = i & 63;
+      float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+      for (int ch = 0; ch < d / 8; ++ch) {
+        uint4 raw = *reinterpret_cast<const uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(f, ch & 7));
+        const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float2 ww = __bfloat1622float2(w2[q]);
+          a0 = fmaf(X.qf[r][ch * 8 + 2 * q], ww.x, a0);
+          a1 = fmaf(X.qf[r][ch * 8 + 2 * q + 1], ww.y, a1);
+        }
+      }
+      X.u_s[r][f] = a0 + a1;
+    }
+    tc::named_bar_sync(2, 256);
+    // phi(q), its normaliser phi(q) . s and q . k_new
+    if (gw < g) {
+      const int r = gw;
+      float u0 = X.u_s[r][lane], u1 = X.u_s[r][lane + 32];
+      float p0, p1, n0, n1;
+      if (L.phi_kind == 1) {
+        p0 = expf(u0); p1 = expf(u1); n0 = expf(-u0); n1 = expf(-u1);
+      } else {
+        float mx = warp_max(fmaxf(u0, u1)), mn = warp_min(fminf(u0, u1));
+        p0 = expf(u0 - mx); p1 = expf(u1 - mx); n0 = expf(mn - u0); n1 = expf(mn - u1);
+        float s1 = warp_sum(p0 + p1), s2 = warp_sum(n0 + n1);
+        p0 /= s1; p1 /= s1; n0 /= s2; n1 /= s2;
+      }
+      float vals[4] = {round_bf16f(p0), round_bf16f(p1), round_bf16f(n0), round_bf16f(n1)};
+      int js[4] = {lane, lane + 32, 64 + lane, 96 + lane};
+      float ld = 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int j = js[q];
+        X.phiq_f[r][j] = vals[q];
+        *reinterpret_cast<T*>(sm + S::phiq + (j >> 6) * 2048 + tc::sw128_off(r, (j & 63) >> 3) + (j & 7) * 2) = __float2bfloat16_rn(vals[q]);
+        ld = fmaf(vals[q], L.s[(size_t)unit * D + j], ld);
+      }
+      ld = warp_sum(ld);
+      float zz = 0.f;
+      for (int j = lane; j < d; j += 32) zz = fmaf(X.qf[r][j], X.knew[j], zz);
+      zz = warp_sum(zz);
+      if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * sl2; }
+    }
+    // H (fp32 [D][d], staged in the buffers of stage 1) -> bf16 H^T, K-major: row c, 64 j per 128-byte row,
+    // two j blocks.  A thread gathers 8 consecutive j of one column c (lanes = consecutive columns: no conflicts).
+    ok = tc::mbar_wait(bar_h, 0, abw) && ok;
+    for (int i = gtid; i < d * (D / 8); i += 256) {
+      const int cc = i % d, jc = i / d;
+      const float* src = reinterpret_cast<const float*>(sm + S::stage0 + S::stage_bytes + ((jc >> 3) ? S::st_v : S::st_k)) + ((jc & 7) * 8) * d + cc;
+      float f8[8];
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) f8[jj] = src[jj * d];
+      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
+    }
+    tc::fence_async_smem();
+    tc::mbar_arrive(bar_ht);
+
+    float lpart[QH], m_prev[QR];
+#pragma unroll
+    for (int r = 0; r < QR; ++r) m_prev[r] = 0.f;
+#pragma unroll
+    for (int r = 0; r < QH; ++r) lpart[r] = 0.f;
+    for (int tile = 0; tile < NT; ++tile) {
+      const int i = tile & 1;
+      const int R = tile * 128 + t;
+      const bool is_g = R < lam;
+      const int slot = R - lam;
+      const bool scored = is_g || slot == s_ev;
+      const int pos = is_g ? L.gpos[(size_t)unit * lam + R] : pos_ev;
+      const uint8_t* vtile = sm + S::stage0 + (size_t)i * S::stage_bytes + S::st_v;
+      uint8_t* ptile = sm + stage_pt(i);
+
+      ok = tc::mbar_wait(bar_vfull(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+      ok = tc::mbar_wait(bar_p, (uint32_t)tile & 1u, abw) && ok;
+      tc::fence_after_sync();
+      // ---- Eq. 10: this thread's half of the value columns
+      float score;
+      {
+        float dn[2];
+        tc::tmem_ld2(tm_p + lane_addr + d, dn);
+        const float den = dn[0] + dn[1];
+        const float inv = den > 0.f ? 1.0f / den : 0.f;
+        // packed pairs: d = v - P / den, four running sums of squares (columns 4k, 4k+1 | 4k+2, 4k+3)
+        const uint64_t ninv2 = tc::pack_f2(-inv, -inv);
+        uint64_t accA = tc::pack_f2(0.f, 0.f), accB = accA;
+#pragma unroll
+        for (int c0 = 0; c0 < HC; c0 += 32) {
+          uint32_t p[32];
+          tc::tmem_ld32u(tm_p + lane_addr + hf * HC + c0, p);
+          if (c0 + 32 >= HC) {                 // [P | den] is read: the next tile's product may overwrite it
+            tc::fence_before_sync();
+            tc::mbar_arrive(bar_pfree);
+          }
+#pragma unroll
+          for (int q8 = 0; q8 < 4; ++q8) {
+            const int cc = hf * HC + c0 + q8 * 8;
+            const uint4 raw = *reinterpret_cast<const uint4*>(vtile + (cc >> 6) * 16384 + tc::sw128_off(t, (cc & 63) >> 3));
+            const uint64_t d01 = tc::fma2(tc::pack_u2(p[q8 * 8 + 0], p[q8 * 8 + 1]), ninv2, tc::pack_u2(raw.x << 16, raw.x & 0xffff0000u));
+            const uint64_t d23 = tc::fma2(tc::pack_u2(p[q8 * 8 + 2], p[q8 * 8 + 3]), ninv2, tc::pack_u2(raw.y << 16, raw.y & 0xffff0000u));
+            const uint64_t d45 = tc::fma2(tc::pack_u2(p[q8 * 8 + 4], p[q8 * 8 + 5]), ninv2, tc::pack_u2(raw.z << 16, raw.z & 0xffff0000u));
+            const uint64_t d67 = tc::fma2(tc::pack_u2(p[q8 * 8 + 6], p[q8 * 8 + 7]), ninv2, tc::pack_u2(raw.w << 16, raw.w & 0xffff0000u));
+            accA = tc::fma2(d01, d01, accA);
+            accB = tc::fma2(d23, d23, accB);
+            accA = tc::fma2(d45, d45, accA);
+            accB = tc::fma2(d67, d67, accB);
+          }
+        }
+        float a0, a1, a2, a3;
+        tc::unpack_f2(accA, a0, a1);
+        tc::unpack_f2(accB, a2, a3);
+        const float ss = (a0 + a1) + (a2 + a3);
+        if (hf == 1) X.ssp[t] = ss;
+        tc::named_bar_sync(2, 256);
+        score = sqrtf(ss + X.ssp[t]);           // hf = 1 threads double their own half; they do not use the score
+      }
+      // lowest score of the tile (ties: the younger pair), and the two lowest values
+      unsigned long long key = ~0ull;
+      if (hf == 0) {
+        if (scored && ok) scu[is_g ? R : lam] = score;
+        if (scored) key = ((unsigned long long)__float_as_uint(score) << 32) | (unsigned)(0x7fffffff - pos);
+        // scores are norms (>= 0): their bit patterns order like unsigned integers
+        const unsigned sb = scored ? __float_as_uint(score) : 0xffffffffu;
+        const unsigned smin = __reduce_min_sync(0xffffffffu, sb);
+        const unsigned tb_ = (sb == smin && scored) ? (unsigned)(0x7fffffff - pos) : 0xffffffffu;
+        const unsigned tmin = __reduce_min_sync(0xffffffffu, tb_);
+        const unsigned long long k = scored || smin != 0xffffffffu ? (((unsigned long long)smin << 32) | tmin) : ~0ull;
+        const bool is_min = scored && sb == smin && tb_ == tmin;
+        const unsigned s2 = __reduce_min_sync(0xffffffffu, is_min ? 0xffffffffu : sb);
+        const float a1 = smin == 0xffffffffu ? CUDART_INF_F : __uint_as_float(smin);
+        const float a2 = s2 == 0xffffffffu ? CUDART_INF_F : __uint_as_float(s2);
+        if (lane == 0) { X.redkey[wq] = k; X.red12[wq][0] = a1; X.red12[wq][1] = a2; }
+      }
+      tc::named_bar_sync(2, 256);
+      unsigned long long tkey = X.redkey[0];
+#pragma unroll
+      for (int w = 1; w < 4; ++w) tkey = X.redkey[w] < tkey ? X.redkey[w] : tkey;
+      // the row left out of O^T: both threads of the row know it from the row's position
+      const unsigned long long rowkey_lo = (unsigned)(0x7fffffff - pos);
+      const bool left_out = scored && (unsigned)tkey == (unsigned)rowkey_lo && tkey != ~0ull;
+      if (left_out) {
+        if (hf == 0) {
+          float a1 = X.red12[0][0], a2 = X.red12[0][1];
+#pragma unroll
+          for (int w = 1; w < 4; ++w) {
+            float b1 = X.red12[w][0], b2 = X.red12[w][1];
+            float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
+            a2 = fminf(hi, fminf(a2, b2));
+            a1 = lo;
+          }
+          X.cand_key[tile] = key;
+          X.cand_score[tile] = score;
+          X.cand_min2[tile] = a2;
+          X.cand_row[tile] = R;
+#pragma unroll
+          for (int r = 0; r < QR; ++r) X.cand_z[tile][r] = X.z_s[i][r][t];
+        } else {
+#pragma unroll
+          for (int ch = 0; ch < d / 8; ++ch)
+            X.cand_v[tile][ch] = *reinterpret_cast<const uint4*>(vtile + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
+        }
+      }
+      if (__any_sync(0xffffffffu, left_out)) {       // its feature row, read back from tensor memory (this thread's half)
+        uint32_t pr[32];
+        tc::tmem_ld32u(tm_phi(i) + lane_addr + hf * 32, pr);
+        if (left_out) {
+          uint32_t* dst = reinterpret_cast<uint32_t*>(&X.cand_phi[tile][0]) + hf * 32;
+#pragma unroll
+          for (int q = 0; q < 32; ++q) dst[q] = pr[q];
+        }
+      }
+      // sums of the weights the feature group wrote (the row left out gives its weights back)
+      if (X.moved[i][0] | X.moved[i][1]) {           // uniform over the block: some row's maximum grew
+        float alpha[QR];
+#pragma unroll
+        for (int r = 0; r < QR; ++r) {
+          const float mt = X.m_s[i][r];
+          alpha[r] = tc::fast_exp2(m_prev[r] - mt);
+          m_prev[r] = mt;
+        }
+#pragma unroll
+        for (int r = 0; r < QH; ++r) lpart[r] *= hf ? alpha[QH + r] : alpha[r];
+        if (hf == 0) {
+          // O^T so far (the products up to the tile before, or the linear term) moves to the new maximum
+          ok = tc::mbar_wait(bar_o(tile & 1), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+          tc::fence_after_sync();
+          float ov[8];
+          tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+          for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
+          tc::tmem_st8(tm_o + lane_addr, ov);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < QH; ++r) {
+        const int rr = hf * QH + r;
+        unsigned short* wp = reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2);
+        if (left_out) *wp = 0;
+        else lpart[r] += __uint_as_float((uint32_t)(*wp) << 16);
+      }
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      tc::mbar_arrive(bar_ptready(i));
+    }
+#pragma unroll
+    for (int r = 0; r < QH; ++r) {
+      float ls = warp_sum(lpart[r]);
+      if (lane == 0) X.l_s[wq][hf * QH + r] = ls;
+    }
+  }
+
+  // ---- all products are complete (the thread that issued the last one has seen it complete)
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const bool okb = X.abort_word == 0;
+  float* opart = reinterpret_cast<float*>(sm + S::stage0 + S::st_v);   // [128][QR]
+  if (warp < 4) {
+    float ov[8];
+    tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+    for (int r = 0; r < QR; ++r) opart[t * QR + r] = ov[r];
+  }
+  // ---- the pair to fold: lowest (score, then youngest) over the tiles' left-out rows
+  int lt = 0;
+  {
+    unsigned long long best = X.cand_key[0];
+    for (int i = 1; i < NT; ++i)
+      if (X.cand_key[i] < best) { best = X.cand_key[i]; lt = i; }
+  }
+  if (warp < g) {                                 // phi(q) . phi_fold
+    const int r = warp;
+    const __nv_bfloat16* pf = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
+    float a = 0.f;
+    for (int j = lane; j < D; j += 32) a = fmaf(X.phiq_f[r][j], __bfloat162float(pf[j]), a);
+    a = warp_sum(a);
+    if (lane == 0) X.dotL[r] = a;
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
+  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
+
+  // ---- Eq. 13: H += phi_fold v_fold^T, s += phi_fold (fp32 additions performed at the L2, no read-back)
+  if (okb) {
+    float* Hgw = L.H + (size_t)unit * D * d;
+    constexpr int per_row = d / 4;
+#pragma unroll 4
+    for (int i = tid; i < D * per_row; i += kDec2Threads) {
+      const int j = i / per_row, c4 = (i % per_row) * 4;
+      const float pj = __bfloat162float(phiL[j]);
+      const uint2 vv = *reinterpret_cast<const uint2*>(vL + c4);
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Hgw + (size_t)i * 4), "f"(pj * bf16lo_f(vv.x)),
+                   "f"(pj * bf16hi_f(vv.x)), "f"(pj * bf16lo_f(vv.y)), "f"(pj * bf16hi_f(vv.y))
+                   : "memory");
+    }
+    if (tid < D) atomicAdd(L.s + (size_t)unit * D + tid, __bfloat162float(phiL[tid]));
+  }
+
+  // ---- Eq. 14: thread (query row r, value column cc)
+  if (okb) {
+    const int il = (NT - 1) & 1;
+    for (int i = tid; i < g * d; i += kDec2Threads) {
+      const int r = i / d, cc = i % d;
+      const float m0 = X.m_s[il][r];
+      const float mf = fmaxf(m0, X.zn[r]);
+      const float a0 = tc::fast_exp2(m0 - mf);
+      float l0 = 0.f;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) l0 += X.l_s[w][r];
+      float num = a0 * opart[cc * QR + r];
+      float den = a0 * l0;
+      for (int ti = 0; ti < NT; ++ti) {
+        if (ti == lt || X.cand_key[ti] == ~0ull) continue;
+        const float p = round_bf16f(tc::fast_exp2(X.cand_z[ti][r] - mf));
+        num = fmaf(p, __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[ti][0])[cc]), num);
+        den += p;
+      }
+      const float pn = tc::fast_exp2(X.zn[r] - mf);
+      num = fmaf(pn, X.vnew[cc], num);
+      den += pn;
+      const float e = tc::fast_exp2(-mf);
+      num = fmaf(e * X.dotL[r], __bfloat162float(vL[cc]), num);
+      den = fmaf(e, X.lden[r] + X.dotL[r], den);
+      ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
+    }
+  }
+
+  // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself)
+  const int rowL = X.cand_row[lt];
+  const T* ring_k = (const T*)L.wk + ((size_t)unit * eta + s_ev) * d;
+  const T* ring_v = (const T*)L.wv + ((size_t)unit * eta + s_ev) * d;
+  if (okb && rowL < lam) {
+    constexpr int nch = d / 8;
+    if (tid < 2 * nch) {
+      const T* src = tid < nch ? ring_k : ring_v;
+      T* dst = (tid < nch ? (T*)L.gk : (T*)L.gv) + ((size_t)unit * lam + rowL) * d;
+      const int ch = tid % nch;
+      *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
+    }
+    if (tid == 64) {
+      L.gpos[(size_t)unit * lam + rowL] = pos_ev;
+      scu[rowL] = scu[lam];
+    }
+  }
+  if (tid == 96 && okb) {
+    // lowest kept / highest folded score of this update
+    float second = X.cand_min2[lt];
+    for (int i = 0; i < NT; ++i)
+      if (i != lt) second = fminf(second, X.cand_score[i]);
+    L.thr[(size_t)unit * 2 + 0] = second;
+    L.thr[(size_t)unit * 2 + 1] = X.cand_score[lt];
+  }
+  __syncthreads();
+  // ---- the new pair enters the window ring
+  if (okb) {
+    constexpr int nch = d / 8;
+    if (tid < 2 * nch) {
+      const T* src = (tid < nch ? (const T*)c.k : (const T*)c.v) + ((size_t)b * L.Hkv + h) * d;
+      T* dst = (tid < nch ? (T*)L.wk : (T*)L.wv) + ((size_t)unit * eta + s_ev) * d;
+      const int ch = tid % nch;
+      *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
+    }
+  }
+  if (!okb && tid == 0) atomicOr(L.status, 8);
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, 512);
+}
+
+}  // namespace lola

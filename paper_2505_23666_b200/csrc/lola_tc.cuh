@@ -261,6 +261,23 @@ __device__ __forceinline__ void tmem_ld32u(uint32_t taddr, uint32_t (&v)[32]) {
                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]) : "r"(taddr) : "memory");
 }
 
+// raw 32-bit: 64 consecutive columns (two loads, one wait)
+__device__ __forceinline__ void tmem_ld64u(uint32_t taddr, uint32_t (&r)[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
+      "tcgen05.wait::ld.sync.aligned;\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr), "r"(taddr + 32u)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, float (&v)[4]) {
+  uint32_t r0, r1, r2, r3;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n\ttcgen05.wait::ld.sync.aligned;\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(taddr) : "memory");
+  v[0] = __uint_as_float(r0); v[1] = __uint_as_float(r1); v[2] = __uint_as_float(r2); v[3] = __uint_as_float(r3);
+}
+
 // named barrier over `count` threads (ids 1..15; 0 is __syncthreads)
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -270,6 +287,65 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// ---- packed fp32 pairs (one instruction works on two values) ------------------------------------
+__device__ __forceinline__ uint64_t pack_f2(float a, float b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ uint64_t pack_u2(uint32_t a, uint32_t b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b)); return r; }
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+__device__ __forceinline__ float min3(float a, float b, float c) { float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+
+// One half of the feature map (Eq. 6) of one row: 64 pre-activations u (raw fp32 bits) -> 64 bf16
+// values as 32 packed pairs.  NEG = false: softmax(u), NEG = true: softmax(-u); exp_kind: exp(+-u)
+// without the normalisation.  Four running sums (elements 4k, 4k+1, 4k+2, 4k+3), added pairwise.
+template <bool NEG>
+__device__ __forceinline__ void phi_half_packed(const uint32_t (&u)[64], bool exp_kind, uint32_t (&out)[32]) {
+  constexpr float kL = NEG ? -1.4426950408889634f : 1.4426950408889634f;
+  float mm = 0.f;
+  if (!exp_kind) {
+    float a = __uint_as_float(u[0]), b = __uint_as_float(u[1]);
+#pragma unroll
+    for (int q = 2; q < 62; q += 4) {
+      a = NEG ? min3(a, __uint_as_float(u[q]), __uint_as_float(u[q + 1])) : max3(a, __uint_as_float(u[q]), __uint_as_float(u[q + 1]));
+      b = NEG ? min3(b, __uint_as_float(u[q + 2]), __uint_as_float(u[q + 3])) : max3(b, __uint_as_float(u[q + 2]), __uint_as_float(u[q + 3]));
+    }
+    a = NEG ? min3(a, __uint_as_float(u[62]), __uint_as_float(u[63])) : max3(a, __uint_as_float(u[62]), __uint_as_float(u[63]));
+    mm = (NEG ? fminf(a, b) : fmaxf(a, b)) * kL;          // = max over the row of u * kL
+  }
+  // packed f32x2 instructions: half the instructions of the plain forms (each thread's instruction
+  // stream, not the pipes, bounds this phase)
+  const uint64_t sc2 = pack_f2(kL, kL), off2 = pack_f2(-mm, -mm);
+  uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = acc0;
+  uint64_t e2[32];
+#pragma unroll
+  for (int q = 0; q < 32; q += 2) {
+    float x0, x1, x2, x3;
+    unpack_f2(fma2(pack_u2(u[2 * q], u[2 * q + 1]), sc2, off2), x0, x1);
+    unpack_f2(fma2(pack_u2(u[2 * q + 2], u[2 * q + 3]), sc2, off2), x2, x3);
+    e2[q] = pack_f2(fast_exp2(x0), fast_exp2(x1));
+    e2[q + 1] = pack_f2(fast_exp2(x2), fast_exp2(x3));
+    acc0 = add2(acc0, e2[q]);
+    acc1 = add2(acc1, e2[q + 1]);
+  }
+  float inv = 1.0f;
+  if (!exp_kind) {
+    float s0, s1, s2, s3;
+    unpack_f2(acc0, s0, s1);
+    unpack_f2(acc1, s2, s3);
+    inv = 1.0f / ((s0 + s1) + (s2 + s3));
+  }
+  const uint64_t inv2 = pack_f2(inv, inv);
+#pragma unroll
+  for (int q = 0; q < 32; ++q) {
+    float lo, hi;
+    unpack_f2(exp_kind ? e2[q] : mul2(e2[q], inv2), lo, hi);
+    __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
+    out[q] = *reinterpret_cast<uint32_t*>(&pr);
+  }
 }
 
 // 8 fp32 -> 8 bf16 packed in a uint4 (element 0 in the low half of x)

@@ -70,6 +70,21 @@ def test_fused_decode_group_sizes(g, batch):
     assert summ["resyncs"] <= 2, summ
 
 
+def test_fused_decode_long_unit():
+    """A unit of more than 8 row tiles (lambda + window > 1024) takes the two-row-group generation kernel."""
+    wl = small_case("fused_long", batch=1, n_q_heads=4, n_kv_heads=2, head_dim=128, feat_half=64, tokens=1280,
+                    chunk=64, window=64, sparse=1088, dtype="bf16", seed=19, decode_steps=12)
+    ls = Lockstep(wl, threads=1)
+    t = 0
+    while t < wl.tokens:
+        ls.prefill(t, wl.chunk, want_out=False, check_state=(t + wl.chunk >= wl.tokens))
+        t += wl.chunk
+    for sidx in range(wl.decode_steps):
+        ls.decode(sidx)
+    summ = ls.summary()
+    assert summ["resyncs"] <= 2, summ
+
+
 def test_cfg3_shape_decode_sample():
     """Two batch rows of the decode workload at its full shapes (lambda 832, window 64, 4 query heads per KV
     head, d 128) after a shortened prefill that fills both caches, 48 fused steps against the oracle."""
