@@ -159,21 +159,29 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     if (lane == 0) {
       const uint32_t idesc_s = tc::make_idesc_bf16(128, 128, false, false);
       const uint32_t idesc_pv = tc::make_idesc_bf16(128, d, false, true);
+      // operand descriptors once; a K step adds its byte offset / 16 to the address field
+      const uint64_t dq0 = tc::make_desc_sw128(sbase + S::q, 16, 1024), dq1 = tc::make_desc_sw128(sbase + S::q + 32768u, 16, 1024);
+      const uint64_t dk0 = tc::make_desc_sw128(sbase + S::stage0 + S::st_k, 16, 1024);
+      const uint64_t dk1 = tc::make_desc_sw128(sbase + S::stage0 + S::stage_bytes + S::st_k, 16, 1024);
+      const uint64_t dv0 = tc::make_desc_sw128(sbase + S::stage0 + S::st_v, 16384, 1024);
+      const uint64_t dv1 = tc::make_desc_sw128(sbase + S::stage0 + S::stage_bytes + S::st_v, 16384, 1024);
       auto issue_s = [&](int w, int kt) {
-        const uint32_t stage = sbase + S::stage0 + (uint32_t)(kt & 1) * S::stage_bytes;
+        const uint64_t dq = w ? dq1 : dq0, dk = (kt & 1) ? dk1 : dk0;
+        const uint32_t ts = tmem + (uint32_t)w * 128u;
 #pragma unroll
-        for (int ks = 0; ks < d / 16; ++ks)
-          tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
-                          tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                          tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
+        for (int ks = 0; ks < d / 16; ++ks) {
+          const uint64_t off = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+          tc::mma_bf16_ss(ts, dq + off, dk + off, idesc_s, ks > 0);
+        }
         tc::mma_commit(BAR(A2_SFULL + w));
       };
       auto issue_pv = [&](int w, int kt) {
-        const uint32_t stage = sbase + S::stage0 + (uint32_t)(kt & 1) * S::stage_bytes;
+        const uint64_t dv = (kt & 1) ? dv1 : dv0;
+        const uint32_t to = tmem + 256u + (uint32_t)w * 128u, tp = tmem + (uint32_t)w * 128u;
+        const uint32_t acc0 = kt > 0 ? 1u : 0u;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + (uint32_t)(ks >> 2) * 64u + (ks & 3) * 8,
-                          tc::make_desc_sw128(stage + S::st_v + ks * 2048, 16384, 1024), idesc_pv, (kt > 0 || ks > 0) ? 1u : 0u);
+          tc::mma_bf16_ts(to, tp + (uint32_t)(ks >> 2) * 64u + (ks & 3) * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, ks > 0 ? 1u : acc0);
         tc::mma_commit(BAR(A2_ODONE + w));
       };
       ok = WAIT(A2_QFULL, 0) && ok;

@@ -26,6 +26,7 @@ struct Decode2Misc {
   float phiq_f[kDecQ][128];      // phi(q) rounded to bf16, as fp32
   float u_s[kDecQ][64];
   float knew[128], vnew[128];
+  float s_f[128];                // the normaliser state s, fp32
   float zn[kDecQ], lden[kDecQ], dotL[kDecQ];
   float redmax[2][4][kDecQ];
   float m_s[2][kDecQ];           // running maximum after tile t (log2 units)
@@ -107,6 +108,17 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   auto stage_v = [&](int i) { return sbase + S::stage0 + (uint32_t)i * S::stage_bytes + S::st_v; };
   auto stage_pt = [&](int i) { return S::stage0 + (uint32_t)i * S::stage_bytes + S::st_pt; };   // offset from sm
 
+  // everything the prologue needs from global memory is requested first, so that the round trips overlap
+  float pre_s = 0.f, pre_k = 0.f, pre_v = 0.f;
+  uint4 pre_q = make_uint4(0, 0, 0, 0);
+  if (tid < D) pre_s = L.s[(size_t)unit * D + tid];
+  if (tid < 16 * (d / 8) && tid / (d / 8) < g)
+    pre_q = *reinterpret_cast<const uint4*>((const T*)c.q + ((size_t)b * L.Hq + h * g + tid / (d / 8)) * d + (tid % (d / 8)) * 8);
+  if (tid >= 256 && tid < 256 + d) {
+    pre_k = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + (tid - 256));
+    pre_v = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + (tid - 256));
+  }
+
   if (tid == 0) {
     X.abort_word = 0;
     for (int i = 0; i < 17; ++i) {
@@ -135,7 +147,8 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   if (role < 2) {
     // rows d, d+1: s as the sum of two bf16 parts (phi . s_hi + phi . s_lo keeps the fp32 normaliser)
     if (tid < D) {
-      const float sv = L.s[(size_t)unit * D + tid];
+      const float sv = pre_s;
+      X.s_f[tid] = sv;
       const __nv_bfloat16 hi = __float2bfloat16_rn(sv);
       const __nv_bfloat16 lo = __float2bfloat16_rn(sv - __bfloat162float(hi));
       const int ch = (tid & 63) >> 3;
@@ -149,10 +162,9 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
     // query rows: B1 rows 64..79 (rows >= g are zero) and an fp32 copy
     constexpr int per_row = d / 8;
-    for (int i = tid; i < 16 * per_row; i += 512) {
-      const int r = i / per_row, ch = i % per_row;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (r < g) val = *reinterpret_cast<const uint4*>((const T*)c.q + ((size_t)b * L.Hq + h * g + r) * d + ch * 8);
+    if (tid < 16 * per_row) {
+      const int r = tid / per_row, ch = tid % per_row;
+      const uint4 val = pre_q;
       *reinterpret_cast<uint4*>(sm + S::b1 + (ch >> 3) * S::b1_blk + tc::sw128_off(64 + r, ch & 7)) = val;
       if (r < QR) {
         const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&val);
@@ -164,9 +176,9 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
       }
     }
-    if (tid < d) {
-      X.knew[tid] = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + tid);
-      X.vnew[tid] = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + tid);
+    if (tid >= 256 && tid < 256 + d) {
+      X.knew[tid - 256] = pre_k;
+      X.vnew[tid - 256] = pre_v;
     }
     if (tid < kDec2MaxTiles) { X.cand_key[tid] = ~0ull; X.cand_score[tid] = CUDART_INF_F; X.cand_min2[tid] = CUDART_INF_F; X.cand_row[tid] = 0; }
     // zero phi(Q) and both Pr^T tiles
@@ -411,7 +423,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         const int j = js[q];
         X.phiq_f[r][j] = vals[q];
         *reinterpret_cast<T*>(sm + S::phiq + (j >> 6) * 2048 + tc::sw128_off(r, (j & 63) >> 3) + (j & 7) * 2) = __float2bfloat16_rn(vals[q]);
-        ld = fmaf(vals[q], L.s[(size_t)unit * D + j], ld);
+        ld = fmaf(vals[q], X.s_f[j], ld);
       }
       ld = warp_sum(ld);
       float zz = 0.f;
@@ -591,7 +603,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   __syncthreads();
   tc::fence_after_sync();
   const bool okb = X.abort_word == 0;
-  float* opart = reinterpret_cast<float*>(sm + S::stage0 + S::st_v);   // [128][QR]
+  float* opart = reinterpret_cast<float*>(sm + S::stage0 + S::stage_bytes + S::st_v);   // [128][QR], in the free stage 1
   if (warp < 4) {
     float ov[8];
     tc::tmem_ld8(tm_o + lane_addr, ov);
@@ -605,34 +617,38 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     for (int i = 1; i < NT; ++i)
       if (X.cand_key[i] < best) { best = X.cand_key[i]; lt = i; }
   }
+  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
+  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
   if (warp < g) {                                 // phi(q) . phi_fold
     const int r = warp;
-    const __nv_bfloat16* pf = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
     float a = 0.f;
-    for (int j = lane; j < D; j += 32) a = fmaf(X.phiq_f[r][j], __bfloat162float(pf[j]), a);
+    for (int j = lane; j < D; j += 32) a = fmaf(X.phiq_f[r][j], __bfloat162float(phiL[j]), a);
     a = warp_sum(a);
     if (lane == 0) X.dotL[r] = a;
   }
-  tc::fence_before_sync();
-  __syncthreads();
-  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
-  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
-
-  // ---- Eq. 13: H += phi_fold v_fold^T, s += phi_fold (fp32 additions performed at the L2, no read-back)
+  // ---- Eq. 13: H += phi_fold v_fold^T.  The update (fp32 [D][d], the layout of H) is staged in the free
+  // buffers of stage 0 and added to H by bulk reductions: the additions happen at the L2, nothing is read back
   if (okb) {
-    float* Hgw = L.H + (size_t)unit * D * d;
     constexpr int per_row = d / 4;
-#pragma unroll 4
+    float4* dH = reinterpret_cast<float4*>(sm + S::stage0);
     for (int i = tid; i < D * per_row; i += kDec2Threads) {
       const int j = i / per_row, c4 = (i % per_row) * 4;
       const float pj = __bfloat162float(phiL[j]);
       const uint2 vv = *reinterpret_cast<const uint2*>(vL + c4);
-      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Hgw + (size_t)i * 4), "f"(pj * bf16lo_f(vv.x)),
-                   "f"(pj * bf16hi_f(vv.x)), "f"(pj * bf16lo_f(vv.y)), "f"(pj * bf16hi_f(vv.y))
-                   : "memory");
+      dH[i] = make_float4(pj * bf16lo_f(vv.x), pj * bf16hi_f(vv.x), pj * bf16lo_f(vv.y), pj * bf16hi_f(vv.y));
     }
-    if (tid < D) atomicAdd(L.s + (size_t)unit * D + tid, __bfloat162float(phiL[tid]));
+    tc::fence_async_smem();
   }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (okb && tid == 0) {
+    float* Hgw = L.H + (size_t)unit * D * d;
+    constexpr uint32_t half_bytes = (uint32_t)(D * d * 4 / 2);
+    tc::bulk_reduce_add_f32(Hgw, sbase + S::stage0, half_bytes);
+    tc::bulk_reduce_add_f32(Hgw + D * d / 2, sbase + S::stage0 + half_bytes, half_bytes);
+    tc::bulk_commit_group();
+  }
+  if (okb && tid < D) atomicAdd(L.s + (size_t)unit * D + tid, __bfloat162float(phiL[tid]));
 
   // ---- Eq. 14: thread (query row r, value column cc)
   if (okb) {
@@ -700,6 +716,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
   }
   if (!okb && tid == 0) atomicOr(L.status, 8);
+  if (tid == 0) tc::bulk_wait_group_all();         // the bulk reductions have read shared memory and are performed
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tmem, 512);
