@@ -27,6 +27,8 @@ struct Decode2Misc {
   float u_s[kDecQ][64];
   float knew[128], vnew[128];
   float s_f[128];                // the normaliser state s, fp32
+  uint4 ring_kv[2 * 16];         // the pair that leaves the window (key chunks, then value chunks), bf16
+  uint4 new_kv[2 * 16];          // the new pair, bf16
   float zn[kDecQ], lden[kDecQ], dotL[kDecQ];
   float redmax[2][4][kDecQ];
   float m_s[2][kDecQ];           // running maximum after tile t (log2 units)
@@ -114,6 +116,13 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   if (tid < D) pre_s = L.s[(size_t)unit * D + tid];
   if (tid < 16 * (d / 8) && tid / (d / 8) < g)
     pre_q = *reinterpret_cast<const uint4*>((const T*)c.q + ((size_t)b * L.Hq + h * g + tid / (d / 8)) * d + (tid % (d / 8)) * 8);
+  uint4 pre_ring = make_uint4(0, 0, 0, 0), pre_new = pre_ring;
+  if (tid >= 384 && tid < 384 + 2 * (d / 8)) {
+    const int i = tid - 384, ch = i % (d / 8);
+    const bool is_k = i < d / 8;
+    pre_ring = *reinterpret_cast<const uint4*>((is_k ? (const T*)L.wk : (const T*)L.wv) + ((size_t)unit * eta + s_ev) * d + ch * 8);
+    pre_new = *reinterpret_cast<const uint4*>((is_k ? (const T*)c.k : (const T*)c.v) + ((size_t)b * L.Hkv + h) * d + ch * 8);
+  }
   if (tid >= 256 && tid < 256 + d) {
     pre_k = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + (tid - 256));
     pre_v = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + (tid - 256));
@@ -175,6 +184,10 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
           X.qf[r][ch * 8 + 2 * q + 1] = ff.y;
         }
       }
+    }
+    if (tid >= 384 && tid < 384 + 2 * (d / 8)) {
+      X.ring_kv[tid - 384] = pre_ring;
+      X.new_kv[tid - 384] = pre_new;
     }
     if (tid >= 256 && tid < 256 + d) {
       X.knew[tid - 256] = pre_k;
@@ -679,40 +692,31 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
   }
 
-  // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself)
+  // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself) and
+  // the new pair enters the window ring; both were fetched at the start
   const int rowL = X.cand_row[lt];
-  const T* ring_k = (const T*)L.wk + ((size_t)unit * eta + s_ev) * d;
-  const T* ring_v = (const T*)L.wv + ((size_t)unit * eta + s_ev) * d;
-  if (okb && rowL < lam) {
+  if (okb) {
     constexpr int nch = d / 8;
-    if (tid < 2 * nch) {
-      const T* src = tid < nch ? ring_k : ring_v;
+    if (tid < 2 * nch && rowL < lam) {
       T* dst = (tid < nch ? (T*)L.gk : (T*)L.gv) + ((size_t)unit * lam + rowL) * d;
-      const int ch = tid % nch;
-      *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
+      *reinterpret_cast<uint4*>(dst + (tid % nch) * 8) = X.ring_kv[tid];
     }
-    if (tid == 64) {
+    if (tid >= 32 && tid < 32 + 2 * nch) {
+      const int i = tid - 32;
+      T* dst = (i < nch ? (T*)L.wk : (T*)L.wv) + ((size_t)unit * eta + s_ev) * d;
+      *reinterpret_cast<uint4*>(dst + (i % nch) * 8) = X.new_kv[i];
+    }
+    if (tid == 64 && rowL < lam) {
       L.gpos[(size_t)unit * lam + rowL] = pos_ev;
       scu[rowL] = scu[lam];
     }
-  }
-  if (tid == 96 && okb) {
-    // lowest kept / highest folded score of this update
-    float second = X.cand_min2[lt];
-    for (int i = 0; i < NT; ++i)
-      if (i != lt) second = fminf(second, X.cand_score[i]);
-    L.thr[(size_t)unit * 2 + 0] = second;
-    L.thr[(size_t)unit * 2 + 1] = X.cand_score[lt];
-  }
-  __syncthreads();
-  // ---- the new pair enters the window ring
-  if (okb) {
-    constexpr int nch = d / 8;
-    if (tid < 2 * nch) {
-      const T* src = (tid < nch ? (const T*)c.k : (const T*)c.v) + ((size_t)b * L.Hkv + h) * d;
-      T* dst = (tid < nch ? (T*)L.wk : (T*)L.wv) + ((size_t)unit * eta + s_ev) * d;
-      const int ch = tid % nch;
-      *reinterpret_cast<uint4*>(dst + ch * 8) = *reinterpret_cast<const uint4*>(src + ch * 8);
+    if (tid == 96) {
+      // lowest kept / highest folded score of this update
+      float second = X.cand_min2[lt];
+      for (int i = 0; i < NT; ++i)
+        if (i != lt) second = fminf(second, X.cand_score[i]);
+      L.thr[(size_t)unit * 2 + 0] = second;
+      L.thr[(size_t)unit * 2 + 1] = X.cand_score[lt];
     }
   }
   if (!okb && tid == 0) atomicOr(L.status, 8);

@@ -158,35 +158,10 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     if (lead && tile + 2 < tile1) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
     {
       tc::named_bar_sync(3 + wg, 512);
-      float e[64];
-      tc::tmem_ld64(tm_a + lane_addr, e);
-      const float sgn = hf ? -kLog2e : kLog2e;
-      if (L.phi_kind == 1) {
-#pragma unroll
-        for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
-      } else {
-        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
-#pragma unroll
-        for (int i = 0; i < 64; i += 4) {
-          m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn);
-          m2 = fmaxf(m2, e[i + 2] * sgn); m3 = fmaxf(m3, e[i + 3] * sgn);
-        }
-        const float mm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-        for (int i = 0; i < 64; i += 4) {
-          e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
-          e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
-          e[i + 2] = tc::fast_exp2(fmaf(e[i + 2], sgn, -mm)); s2 += e[i + 2];
-          e[i + 3] = tc::fast_exp2(fmaf(e[i + 3], sgn, -mm)); s3 += e[i + 3];
-        }
-        const float inv = 1.0f / ((s0 + s1) + (s2 + s3));
-#pragma unroll
-        for (int i = 0; i < 64; ++i) e[i] *= inv;
-      }
-      uint32_t pk2[32];
-#pragma unroll
-      for (int i = 0; i < 32; ++i) pk2[i] = pack_bf16x2(e[2 * i], e[2 * i + 1]);
+      uint32_t u[64], pk2[32];
+      tc::tmem_ld64u(tm_a + lane_addr, u);
+      if (hf) tc::phi_half_packed<true>(u, L.phi_kind == 1, pk2);
+      else tc::phi_half_packed<false>(u, L.phi_kind == 1, pk2);
       tc::tmem_st32u(tm_phi + lane_addr + hf * 32, pk2);
       if (wg == 0) asm volatile("bar.arrive 4, 512;" ::: "memory"); else asm volatile("bar.arrive 3, 512;" ::: "memory");
     }

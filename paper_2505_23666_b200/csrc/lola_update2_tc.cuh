@@ -312,42 +312,15 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   else { ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1; }
   tc::fence_after_sync();
   if (tid < 256) {                                                   // one thread pair per row: half of the feature map each
-    float e[64];
-    tc::tmem_ld64(tm_u + lane_addr, e);
-    const float sgn = hf ? -kLog2e : kLog2e;
-    if (L.phi_kind == 1) {
-#pragma unroll
-      for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
-    } else {
-      float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
-#pragma unroll
-      for (int i = 0; i < 64; i += 4) {
-        m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn);
-        m2 = fmaxf(m2, e[i + 2] * sgn); m3 = fmaxf(m3, e[i + 3] * sgn);
-      }
-      const float mm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-      for (int i = 0; i < 64; i += 4) {
-        e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
-        e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
-        e[i + 2] = tc::fast_exp2(fmaf(e[i + 2], sgn, -mm)); s2 += e[i + 2];
-        e[i + 3] = tc::fast_exp2(fmaf(e[i + 3], sgn, -mm)); s3 += e[i + 3];
-      }
-      const float inv = 1.0f / ((s0 + s1) + (s2 + s3));
-#pragma unroll
-      for (int i = 0; i < 64; ++i) e[i] *= inv;
-    }
+    uint32_t u[64], pk2[32];
+    tc::tmem_ld64u(tm_u + lane_addr, u);
+    if (hf) tc::phi_half_packed<true>(u, L.phi_kind == 1, pk2);
+    else tc::phi_half_packed<false>(u, L.phi_kind == 1, pk2);
     // phi tile over the key tile (consumed): row = folded pair, 64 features per 128-byte row and block
 #pragma unroll
-    for (int ch = 0; ch < 8; ++ch) {
-      uint4 o;
-      o.x = pack_bf16x2(e[ch * 8], e[ch * 8 + 1]);
-      o.y = pack_bf16x2(e[ch * 8 + 2], e[ch * 8 + 3]);
-      o.z = pack_bf16x2(e[ch * 8 + 4], e[ch * 8 + 5]);
-      o.w = pack_bf16x2(e[ch * 8 + 6], e[ch * 8 + 7]);
-      *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t, ch)) = o;
-    }
+    for (int ch = 0; ch < 8; ++ch)
+      *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t, ch)) =
+          make_uint4(pk2[ch * 4], pk2[ch * 4 + 1], pk2[ch * 4 + 2], pk2[ch * 4 + 3]);
   }
   asm volatile("cp.async.wait_all;" ::: "memory");
   tc::fence_async_smem();
