@@ -247,22 +247,26 @@ inline bool fast_update_path(const lola_state* st, const Call& c) {
 // memories (scores, positions) and write scores / work lists, so they may run beside the attention
 // kernel on another stream.
 template <int DPL>
-int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss) {
+int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss, int busy_sms = 0) {
   const Layer& L = st->L;
   const int U = L.B * L.Hkv;
   const int NT = (c.count_g / 64 + (L.eta + 63) / 64 + 1) / 2;
   int tpc = (U * NT + 147) / 148;
   tpc = std::max(2, tpc + (tpc & 1));
+  // beside the attention kernel (one block per SM, busy_sms of them) the blocks of this kernel should fit
+  // the SMs that are left in one round: a second round would end after the attention kernel does
+  if (busy_sms > 0 && busy_sms < 148) {
+    const int avail = 148 - busy_sms;
+    int t2 = tpc;
+    while (t2 < NT && U * ((NT + t2 - 1) / t2) > avail) ++t2;
+    if (U * ((NT + t2 - 1) / t2) <= avail) tpc = t2;
+  }
   const uint4* img = (const uint4*)(st->base + st->lay.wt);
   __nv_bfloat16* himg = (__nv_bfloat16*)(st->base + st->lay.himg);
-  {
-    LaunchScope scope(st, LOLA_KERNEL_SCORE, ss);
-    dim3 grid((NT + tpc - 1) / tpc, U);
-    k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
-    if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
-  }
-  LaunchScope scope(st, LOLA_KERNEL_SELECT, ss);
-  k_update2_tc<DPL, 1><<<U, kUp2Threads, sizeof(Update2Misc) + 1024, ss>>>(L, c, img, himg);
+  // the selection (Eq. 12) runs in the scoring kernel: the last block of a unit to finish does it
+  LaunchScope scope(st, LOLA_KERNEL_SCORE, ss);
+  dim3 grid((NT + tpc - 1) / tpc, U);
+  k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
@@ -327,7 +331,7 @@ int run_prefill(lola_state* st, Call c, cudaStream_t s) {
       return LOLA_ERR_CUDA;
     // scoring and selection are enqueued first: their many short CTAs take the SMs at once and the
     // attention CTAs fill in as they drain; the fold joins both
-    rc = launch_score_select<DPL>(st, c, st->aux);
+    rc = launch_score_select<DPL>(st, c, st->aux, (((st->L.g + 1) / 2 + 1) / 2) * st->L.B * st->L.Hkv);
     if (rc != LOLA_OK) return rc;
     rc = launch_attend<T, DPL>(st, c, s);
     if (rc != LOLA_OK) return rc;

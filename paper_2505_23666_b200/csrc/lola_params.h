@@ -29,7 +29,7 @@ struct Layer {          // fixed for the life of a state
   int* fold_idx;        // [U, cmax] E-indices of the pairs to fold
   int* move_src;        // [U, cmax] index (into the leaving pairs) of each pair entering G
   int* move_dst;        // [U, cmax] slot it goes to
-  int* counts;          // [U, 4]: n_fold, n_move, (unused), (unused)
+  int* counts;          // [U, 4]: n_fold, n_move, scoring blocks that have finished (0 between calls), (unused)
   float* thr;           // [U, 2]
   int* status;          // [1]
   const void* W;        // [Hkv, d, F]

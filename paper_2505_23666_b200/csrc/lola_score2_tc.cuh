@@ -14,6 +14,7 @@
 #include <cuda.h>
 
 #include "lola_decode_tc.cuh"
+#include "lola_update2_tc.cuh"
 #include "lola_generic.cuh"
 #include "lola_tc.cuh"
 
@@ -212,8 +213,22 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   }
   if (!ok && (tid & 255) == 0) atomicOr(L.status, 16);
   tc::fence_before_sync();
+  __threadfence();                                   // this block's scores are visible before it counts itself
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tmem, 512);
+  // ---- the last block of a unit to finish selects the pairs to fold (Eq. 12) from all the unit's scores
+  __shared__ int is_last;
+  if (tid == 0) {
+    int* arrived = L.counts + (size_t)unit * 4 + 2;
+    const int prev = atomicAdd(arrived, 1);
+    is_last = prev == (int)gridDim.x - 1;
+    if (is_last) *arrived = 0;                       // ready for the next call
+  }
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    update2_body<DPL, 1>(L, c, wt_image, nullptr, sm, unit);
+  }
 }
 
 }  // namespace lola

@@ -55,22 +55,23 @@ static_assert(sizeof(Update2Misc) <= 2 * kUp2MaxE * 4 + 8192, "misc region too s
 
 // PHASE 1: selection only (steps 1-2; the lists go to the state's work-list arrays, so it can run beside
 // the attention kernel, which only reads the memories).  PHASE 2: steps 3-4 from those lists.
+// The body works on one unit with a block of kUp2Threads threads and `sm`, 1024-byte aligned dynamic shared
+// memory (PHASE 1 needs sizeof(Update2Misc) bytes of it, the others Update2Smem<DPL>::total); the scoring
+// kernel runs PHASE 1 in its last block of a unit.
 template <int DPL, int PHASE>
-__global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image, __nv_bfloat16* ht_image) {
+__device__ __forceinline__ void update2_body(const Layer& L, const Call& c, const uint4* wt_image, __nv_bfloat16* ht_image,
+                                             uint8_t* sm, const int unit) {
   using S = Update2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
   constexpr int D = 128;
   constexpr int nch = d / 8;
-  constexpr float kLog2e = 1.4426950408889634f;
   typedef __nv_bfloat16 T;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = tc::smem_u32(sm);
   constexpr uint32_t kMisc = PHASE == 1 ? 0u : S::misc;          // the selection needs the small arrays only
   Update2Misc& X = *reinterpret_cast<Update2Misc*>(sm + kMisc);
 
-  const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
+  const int b = unit / L.Hkv, h = unit % L.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lam = L.lam, eta = L.eta;
   // PHASE 2 also serves calls that fold nothing (nothing leaves the window yet, or every leaving pair
@@ -394,6 +395,13 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   tc::fence_before_sync();
   __syncthreads();
   if (fold && warp == 0) tc::tmem_dealloc(X.tmem_slot, 256);
+}
+
+template <int DPL, int PHASE>
+__global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image, __nv_bfloat16* ht_image) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  update2_body<DPL, PHASE>(L, c, wt_image, ht_image, sm, (int)blockIdx.x);
 }
 
 // Rebuilds the bf16 operand image of H for every unit (after a path that changed H without
