@@ -200,6 +200,23 @@ struct LaunchScope {
   }
 };
 
+// Launch with programmatic stream serialization: the kernel may become resident while the kernel before it
+// in the stream still runs, and waits inside (griddepcontrol.wait) before it touches memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <int DPL>
 int ensure_h_image(lola_state* st, cudaStream_t s) {
   if (st->himg_valid) return LOLA_OK;
@@ -222,10 +239,10 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
       if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
       LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
       dim3 grid2(((L.g + 1) / 2 + 1) / 2, L.B * L.Hkv);
-      k_attend2_tc<DPL><<<grid2, kAt2Threads, Attend2Smem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, tq, tk,
-                                                                            tv, (const uint4*)(st->base + st->lay.wt),
-                                                                            (const __nv_bfloat16*)(st->base + st->lay.himg));
-      return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+      const cudaError_t le = launch_pdl(k_attend2_tc<DPL>, grid2, dim3(kAt2Threads), Attend2Smem<DPL>::bytes, s, L, c, st->tm_gk, st->tm_gv,
+                                        st->tm_wk, st->tm_wv, tq, tk, tv, (const uint4*)(st->base + st->lay.wt),
+                                        (const __nv_bfloat16*)(st->base + st->lay.himg));
+      return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
     }
   }
   LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
@@ -276,9 +293,9 @@ template <int DPL>
 int launch_apply(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
-  k_update2_tc<DPL, 2><<<L.B * L.Hkv, kUp2Threads, Update2Smem<DPL>::bytes, s>>>(
-      L, c, (const uint4*)(st->base + st->lay.wt), (__nv_bfloat16*)(st->base + st->lay.himg));
-  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+  const cudaError_t le = launch_pdl(k_update2_tc<DPL, 2>, dim3(L.B * L.Hkv), dim3(kUp2Threads), Update2Smem<DPL>::bytes, s, L, c,
+                                    (const uint4*)(st->base + st->lay.wt), (__nv_bfloat16*)(st->base + st->lay.himg));
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
 template <typename T, int DPL>
@@ -473,6 +490,27 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       e[6] = cudaFuncSetAttribute(k_decode2_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
     }
     for (int i = 0; i < 7; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
+    // one shared-memory carve-out for the kernels that follow each other in a step: a change of the
+    // carve-out between two launches costs idle time on every SM
+    const int co = (int)cudaSharedmemCarveoutMaxShared;
+    if (cfg->head_dim == 128) {
+      cudaFuncSetAttribute(k_decode_tc<4, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_decode2_tc<4, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_decode2_tc<4, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_score2_tc<4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_update2_tc<4, 2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_attend2_tc<4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+    } else {
+      cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_decode2_tc<2, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_decode2_tc<2, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_score2_tc<2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_update2_tc<2, 2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+      cudaFuncSetAttribute(k_attend2_tc<2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
+    }
+    cudaGetLastError();   // a refused preference is not an error
   }
   if (rc == LOLA_OK && st->have_maps) {
     // host-side objects only (no device memory): a second stream and two events to run the scoring

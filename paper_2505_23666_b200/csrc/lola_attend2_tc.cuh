@@ -98,9 +98,11 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
+  if (tid == 0) tc::grid_dep_launch_dependents();    // the next kernel may set itself up beside this one
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
+  tc::grid_dep_wait();                               // everything before this kernel in the stream is complete
   const uint32_t tmem = X.tmem_slot;
 
   // block `blk` of the key stream -> TMA source

@@ -215,6 +215,11 @@ __device__ __forceinline__ void bulk_reduce_add_f32(float* dst, uint32_t src_sme
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Programmatic dependent launch: a kernel launched with programmatic stream serialization may start
+// while the kernel before it in the stream still runs; it must pass grid_dep_wait() before it touches
+// anything that kernel (or an earlier one) produces or still reads.  Both are no-ops in a normal launch.
+__device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }

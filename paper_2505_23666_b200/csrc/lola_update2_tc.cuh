@@ -89,6 +89,14 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
 
   if (tid == 0) { tc::mbar_init(bar, 1); tc::mbar_init_fence(); X.min_keep = 0xffffffffu; X.n_equal = 0; }
   if (PHASE != 1 && fold && warp == 0) tc::tmem_alloc(&X.tmem_slot, 256);
+  if (PHASE == 2) {
+    // launched early (programmatic dependent launch): the zeroed operand tiles need nothing from memory
+    if (tid == 0) tc::grid_dep_launch_dependents();
+    if (fold)
+      for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
+        *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
+    tc::grid_dep_wait();                             // the attention kernel has read the memories this kernel changes
+  }
   // H of the unit streams into shared memory (asynchronous 16-byte copies) meanwhile
   if (PHASE != 1 && fold) {
     const float* Hg = L.H + (size_t)unit * D * d;
@@ -105,8 +113,9 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   if (PHASE != 1 && fold) {
     const uint4* img = wt_image + (size_t)h * kblk * 512;
     for (int i = tid; i < kblk * 512; i += kUp2Threads) *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
-    for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
-      *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
+    if (PHASE != 2)
+      for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
+        *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
   }
   int nGL = 0, nMove = 0;
   unsigned thr_key = 0;
