@@ -64,6 +64,14 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 
+// The tile loader as a real function: the issuing threads reach it from many places, and every inlined copy
+// would add to an instruction footprint that four different roles already share.
+template <int DPL>
+__device__ __noinline__ void decode2_issue_tile(uint32_t dst, const CUtensorMap* tm_g, const CUtensorMap* tm_w, int tile, int nGB, int nRB,
+                                                int unit, uint32_t bar) {
+  decode_issue_tile<DPL>(dst, tm_g, tm_w, tile, nGB, nRB, unit, bar);
+}
+
 template <int DPL, int QR>
 __global__ void __launch_bounds__(kDec2Threads, 1)
 k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
@@ -144,12 +152,12 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     tc::mbar_expect_tx(bar_w, (uint32_t)kblk * 8192u);
     for (int kb = 0; kb < kblk; ++kb)
       tc::bulk_copy_g2s(sbase + S::b1 + (uint32_t)kb * S::b1_blk, wt_image + ((size_t)h * kblk + kb) * 512, 8192u, bar_w);
-    decode_issue_tile<DPL>(stage_k(0), &tm_gk, &tm_wk, 0, nGB, nRB, unit, bar_kfull(0));
+    decode2_issue_tile<DPL>(stage_k(0), &tm_gk, &tm_wk, 0, nGB, nRB, unit, bar_kfull(0));
     const float* Hg = L.H + (size_t)unit * D * d;
     tc::mbar_expect_tx(bar_h, (uint32_t)(D * d * 4));
     tc::bulk_copy_g2s(stage_k(1), Hg, 64u * d * 4u, bar_h);
     tc::bulk_copy_g2s(stage_v(1), Hg + 64 * d, 64u * d * 4u, bar_h);
-    decode_issue_tile<DPL>(stage_v(0), &tm_gv, &tm_wv, 0, nGB, nRB, unit, bar_vfull(0));
+    decode2_issue_tile<DPL>(stage_v(0), &tm_gv, &tm_wv, 0, nGB, nRB, unit, bar_vfull(0));
   }
 
   // ---- operands that stay for the whole unit (compute warps)
@@ -235,7 +243,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       int next_k = 2;                                  // tiles 0 and 1 are loaded by the prologue
       int n1 = 0;                                      // first products issued so far
       auto load_k = [&]() {
-        decode_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
+        decode2_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
         ++next_k;
       };
       auto poll_k = [&]() {
@@ -281,8 +289,8 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
           ok = tc::mbar_wait(bar_ht, 0, abw) && ok;
           tc::fence_after_sync();
           if (NT > 1) {
-            decode_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
-            decode_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
+            decode2_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
+            decode2_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
           }
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
@@ -320,7 +328,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         const int ev = tile + 1;                                      // completion event of this product
         tc::mma_commit(bar_o(ev & 1));
         ok = tc::mbar_wait(bar_o(ev & 1), (uint32_t)(ev >> 1) & 1u, abw) && ok;
-        if (tile + 2 < NT) decode_issue_tile<DPL>(stage_v(i), &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_vfull(i));
+        if (tile + 2 < NT) decode2_issue_tile<DPL>(stage_v(i), &tm_gv, &tm_wv, tile + 2, nGB, nRB, unit, bar_vfull(i));
       }
     }
     __syncwarp();
@@ -354,8 +362,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       {
         uint32_t u[64];
         tc::tmem_ld64u(tm_uz(i) + lane_addr, u);
-        if (hf) tc::phi_half_packed<true>(u, exp_kind, pk2);
-        else tc::phi_half_packed<false>(u, exp_kind, pk2);
+        tc::phi_half(u, hf != 0, exp_kind, pk2);
       }
       if (tile >= 2) {
         // the buffers of tile - 2: its feature rows and q.k columns were used by the score group, its

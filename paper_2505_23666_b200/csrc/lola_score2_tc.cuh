@@ -161,8 +161,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       tc::named_bar_sync(3 + wg, 512);
       uint32_t u[64], pk2[32];
       tc::tmem_ld64u(tm_a + lane_addr, u);
-      if (hf) tc::phi_half_packed<true>(u, L.phi_kind == 1, pk2);
-      else tc::phi_half_packed<false>(u, L.phi_kind == 1, pk2);
+      tc::phi_half(u, hf != 0, L.phi_kind == 1, pk2);
       tc::tmem_st32u(tm_phi + lane_addr + hf * 32, pk2);
       if (wg == 0) asm volatile("bar.arrive 4, 512;" ::: "memory"); else asm volatile("bar.arrive 3, 512;" ::: "memory");
     }

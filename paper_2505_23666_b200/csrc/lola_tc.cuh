@@ -151,20 +151,25 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // and returns false; the caller records the failure and carries on to its cleanup.  With an abort
 // word (shared memory) the first wait that gives up raises it and every other wait of the CTA that
 // polls it returns false at once, so one lost signal cannot add up to many timeouts.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word = nullptr) {
+// The polling loop is a real function (one copy per kernel): the kernels wait in dozens of places and
+// their instruction footprint matters.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}\n"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word) {
   unsigned long long deadline = 0;
   for (uint32_t it = 0;; ++it) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t"
-        "}\n"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (done) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     if (it > 64) __nanosleep(64);
     if ((it & 255u) == 255u) {
       if (abort_word && *abort_word) return false;
@@ -176,6 +181,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word = nullptr) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_word);
 }
 
 // ---- TMA (bulk tensor copies global -> shared, completion on an mbarrier) ------------------------
@@ -314,36 +323,44 @@ __device__ __forceinline__ float max3(float a, float b, float c) { float d; asm(
 __device__ __forceinline__ float min3(float a, float b, float c) { float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
 
 // One half of the feature map (Eq. 6) of one row: 64 pre-activations u (raw fp32 bits) -> 64 bf16
-// values as 32 packed pairs.  NEG = false: softmax(u), NEG = true: softmax(-u); exp_kind: exp(+-u)
+// values as 32 packed pairs.  neg = false: softmax(u), neg = true: softmax(-u); exp_kind: exp(+-u)
 // without the normalisation.  Four running sums (elements 4k, 4k+1, 4k+2, 4k+3), added pairwise.
-template <bool NEG>
-__device__ __forceinline__ void phi_half_packed(const uint32_t (&u)[64], bool exp_kind, uint32_t (&out)[32]) {
-  constexpr float kL = NEG ? -1.4426950408889634f : 1.4426950408889634f;
+// One instruction stream serves both signs (the sign is data): the two threads of a row run the same
+// code, which keeps the instruction footprint of the kernels small.  Packed f32x2 instructions: half
+// the instructions of the plain forms (each thread's instruction stream, not the pipes, bounds this phase).
+__device__ __forceinline__ void phi_half(const uint32_t (&u)[64], bool neg, bool exp_kind, uint32_t (&out)[32]) {
+  const float kL = neg ? -1.4426950408889634f : 1.4426950408889634f;
+  const uint64_t sc2 = pack_f2(kL, kL);
+  uint64_t x2[32];
+#pragma unroll
+  for (int q = 0; q < 32; ++q) x2[q] = mul2(pack_u2(u[2 * q], u[2 * q + 1]), sc2);   // u * kL, in log2 units
   float mm = 0.f;
   if (!exp_kind) {
-    float a = __uint_as_float(u[0]), b = __uint_as_float(u[1]);
+    float a, b;
+    unpack_f2(x2[0], a, b);
 #pragma unroll
-    for (int q = 2; q < 62; q += 4) {
-      a = NEG ? min3(a, __uint_as_float(u[q]), __uint_as_float(u[q + 1])) : max3(a, __uint_as_float(u[q]), __uint_as_float(u[q + 1]));
-      b = NEG ? min3(b, __uint_as_float(u[q + 2]), __uint_as_float(u[q + 3])) : max3(b, __uint_as_float(u[q + 2]), __uint_as_float(u[q + 3]));
+    for (int q = 1; q < 31; q += 2) {
+      float c0, c1, c2, c3;
+      unpack_f2(x2[q], c0, c1);
+      unpack_f2(x2[q + 1], c2, c3);
+      a = max3(a, c0, c1);
+      b = max3(b, c2, c3);
     }
-    a = NEG ? min3(a, __uint_as_float(u[62]), __uint_as_float(u[63])) : max3(a, __uint_as_float(u[62]), __uint_as_float(u[63]));
-    mm = (NEG ? fminf(a, b) : fmaxf(a, b)) * kL;          // = max over the row of u * kL
+    float c0, c1;
+    unpack_f2(x2[31], c0, c1);
+    mm = fmaxf(max3(a, c0, c1), b);
   }
-  // packed f32x2 instructions: half the instructions of the plain forms (each thread's instruction
-  // stream, not the pipes, bounds this phase)
-  const uint64_t sc2 = pack_f2(kL, kL), off2 = pack_f2(-mm, -mm);
+  const uint64_t off2 = pack_f2(-mm, -mm);
   uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = acc0;
-  uint64_t e2[32];
 #pragma unroll
   for (int q = 0; q < 32; q += 2) {
-    float x0, x1, x2, x3;
-    unpack_f2(fma2(pack_u2(u[2 * q], u[2 * q + 1]), sc2, off2), x0, x1);
-    unpack_f2(fma2(pack_u2(u[2 * q + 2], u[2 * q + 3]), sc2, off2), x2, x3);
-    e2[q] = pack_f2(fast_exp2(x0), fast_exp2(x1));
-    e2[q + 1] = pack_f2(fast_exp2(x2), fast_exp2(x3));
-    acc0 = add2(acc0, e2[q]);
-    acc1 = add2(acc1, e2[q + 1]);
+    float x0, x1, x2f, x3;
+    unpack_f2(add2(x2[q], off2), x0, x1);
+    unpack_f2(add2(x2[q + 1], off2), x2f, x3);
+    x2[q] = pack_f2(fast_exp2(x0), fast_exp2(x1));
+    x2[q + 1] = pack_f2(fast_exp2(x2f), fast_exp2(x3));
+    acc0 = add2(acc0, x2[q]);
+    acc1 = add2(acc1, x2[q + 1]);
   }
   float inv = 1.0f;
   if (!exp_kind) {
@@ -356,10 +373,14 @@ __device__ __forceinline__ void phi_half_packed(const uint32_t (&u)[64], bool ex
 #pragma unroll
   for (int q = 0; q < 32; ++q) {
     float lo, hi;
-    unpack_f2(exp_kind ? e2[q] : mul2(e2[q], inv2), lo, hi);
+    unpack_f2(exp_kind ? x2[q] : mul2(x2[q], inv2), lo, hi);
     __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
     out[q] = *reinterpret_cast<uint32_t*>(&pr);
   }
+}
+template <bool NEG>
+__device__ __forceinline__ void phi_half_packed(const uint32_t (&u)[64], bool exp_kind, uint32_t (&out)[32]) {
+  phi_half(u, NEG, exp_kind, out);
 }
 
 // 8 fp32 -> 8 bf16 packed in a uint4 (element 0 in the low half of x)

@@ -324,8 +324,7 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   if (tid < 256) {                                                   // one thread pair per row: half of the feature map each
     uint32_t u[64], pk2[32];
     tc::tmem_ld64u(tm_u + lane_addr, u);
-    if (hf) tc::phi_half_packed<true>(u, L.phi_kind == 1, pk2);
-    else tc::phi_half_packed<false>(u, L.phi_kind == 1, pk2);
+    tc::phi_half(u, hf != 0, L.phi_kind == 1, pk2);
     // phi tile over the key tile (consumed): row = folded pair, 64 features per 128-byte row and block
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch)
