@@ -241,74 +241,57 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       };
       // key tiles: tile x + 2 streams into the buffer of tile x once that tile's first product is complete
       int next_k = 2;                                  // tiles 0 and 1 are loaded by the prologue
-      int n1 = 0;                                      // first products issued so far
-      auto load_k = [&]() {
-        decode2_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
-        ++next_k;
-      };
-      auto poll_k = [&]() {
-        while (next_k < NT && next_k - 2 < n1 && mbar_test(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u)) load_k();
-      };
-      // waits for a barrier and keeps the key stream going meanwhile
-      auto wait_poll = [&](uint32_t bar, uint32_t parity) {
-        for (uint32_t it = 0; it < 64u; ++it) {
-          uint32_t done;
-          asm volatile(
-              "{\n\t"
-              ".reg .pred p;\n\t"
-              "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-              "selp.u32 %0, 1, 0, p;\n\t"
-              "}\n"
-              : "=r"(done)
-              : "r"(bar), "r"(parity)
-              : "memory");
-          if (done) return true;
-          poll_k();
-        }
-        return tc::mbar_wait(bar, parity, abw);
-      };
-      auto mma1 = [&](int tile) {                      // needs: key tile landed, [U | Z] buffer free
-        while (next_k <= tile) {                       // (its load must have been issued)
-          ok = tc::mbar_wait(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u, abw) && ok;
-          load_k();
-        }
-        ok = wait_poll(bar_kfull(tile & 1), (uint32_t)(tile >> 1) & 1u) && ok;
-        tc::fence_after_sync();
-        issue_mma1(tile);
-        ++n1;
-      };
+      int next1 = 0;                                   // next first product to issue
       ok = tc::mbar_wait(bar_w, 0, abw) && ok;
-      mma1(0);
-      for (int tile = 0; tile < NT; ++tile) {
+      // one copy of every step (iteration -1 only issues the first tile's first product): the code of this
+      // thread shares the instruction cache with the two compute groups
+      for (int tile = -1; tile < NT; ++tile) {
         const int i = tile & 1;
-        ok = wait_poll(bar_phidone(i), (uint32_t)(tile >> 1) & 1u) && ok;   // phi(tile) written, [U | Z] of this tile read
-        tc::fence_after_sync();
-        if (tile == 0) {
-          // H^T is in place: stage 1 is free for the second tile; O^T starts as the linear term
-          // H^T phi(Q)^T, with weight exp(0 - m), m = 0 so far
-          ok = tc::mbar_wait(bar_ht, 0, abw) && ok;
+        if (tile >= 0) {
+          ok = tc::mbar_wait(bar_phidone(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;   // phi(tile) written, [U | Z] of this tile read
           tc::fence_after_sync();
-          if (NT > 1) {
-            decode2_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
-            decode2_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
+          if (tile == 0) {
+            // H^T is in place: stage 1 is free for the second tile; O^T starts as the linear term
+            // H^T phi(Q)^T, with weight exp(0 - m), m = 0 so far
+            ok = tc::mbar_wait(bar_ht, 0, abw) && ok;
+            tc::fence_after_sync();
+            if (NT > 1) {
+              decode2_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
+              decode2_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
+            }
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+              tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
+                              tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc0, ks > 0);
+            tc::mma_commit(bar_o(0));
+          } else {
+            ok = tc::mbar_wait(bar_pfree, (uint32_t)(tile - 1) & 1u, abw) && ok;   // [P | den] of the tile before is read
+            tc::fence_after_sync();
           }
+          const uint32_t tph = tm_phi(i);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
-            tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
-                            tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc0, ks > 0);
-          tc::mma_commit(bar_o(0));
-        } else {
-          ok = wait_poll(bar_pfree, (uint32_t)(tile - 1) & 1u) && ok;   // [P | den] of the tile before is read
-          tc::fence_after_sync();
+            tc::mma_bf16_ts(tm_p, tph + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
+          tc::mma_commit(bar_p);
         }
-        const uint32_t tph = tm_phi(i);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          tc::mma_bf16_ts(tm_p, tph + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
-        tc::mma_commit(bar_p);
-        // first products run two tiles ahead of the feature group: the buffer this tile used is free
-        if (tile == 0 && NT > 1) mma1(1);
-        if (tile + 2 < NT) mma1(tile + 2);
+        // first products run two tiles ahead of the feature group: the buffer a tile used is free once its
+        // feature rows are written (seen above)
+        const int upto = tile < 0 ? 0 : min(tile + 2, NT - 1);
+        for (; next1 <= upto; ++next1) {
+          while (next_k <= next1) {                    // (the tile's load must have been issued)
+            ok = tc::mbar_wait(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u, abw) && ok;
+            decode2_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
+            ++next_k;
+          }
+          ok = tc::mbar_wait(bar_kfull(next1 & 1), (uint32_t)(next1 >> 1) & 1u, abw) && ok;
+          tc::fence_after_sync();
+          issue_mma1(next1);
+        }
+        // key tiles whose buffer is free already (the product that read it is complete) start to stream now
+        while (next_k < NT && next_k - 2 < next1 && mbar_test(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u)) {
+          decode2_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
+          ++next_k;
+        }
       }
     }
     __syncwarp();
