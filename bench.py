@@ -34,24 +34,28 @@ METRIC = "LoLA tokens/s per layer"
 UNIT = "tokens/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch from an ncu capture (profiles/), valid only
-# while the kernel's source is the one that was captured (first 16 hex digits of its SHA-256)
+# while the kernel's sources are the ones that were captured (first 16 hex digits of the SHA-256 over them)
 NCU_TRAFFIC = {
-    "decode": {"source": "paper_2505_23666_b200/csrc/lola_decode_tc.cuh", "sha256_16": "c1075588157eadeb",
-               "bytes_per_launch": 302.6e6, "units": 512},
+    "decode": {"sources": ["paper_2505_23666_b200/csrc/lola_decode2_tc.cuh", "paper_2505_23666_b200/csrc/lola_decode_tc.cuh",
+                           "paper_2505_23666_b200/csrc/lola_tc.cuh"],
+               "sha256_16": "2b54e132152e8690", "bytes_per_launch": 305.1e6, "units": 512},
 }
 
 
 def ncu_traffic(kind, units):
     """DRAM traffic of one launch of the dominant kernel per the committed ncu capture, scaled by the units a
-    launch processes; None when the kernel has changed since the capture."""
+    launch processes; None when the kernel's sources have changed since the capture."""
     import hashlib
     ent = NCU_TRAFFIC.get(kind)
     if not ent:
         return None
     try:
-        with open(os.path.join(ROOT, ent["source"]), "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest()[:16] != ent["sha256_16"]:
-                return None
+        h = hashlib.sha256()
+        for src in ent["sources"]:
+            with open(os.path.join(ROOT, src), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest()[:16] != ent["sha256_16"]:
+            return None
     except OSError:
         return None
     return ent["bytes_per_launch"] * units / ent["units"]
@@ -324,7 +328,7 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         ncores = len(os.sched_getaffinity(0))
-        srows = rows[:min(len(rows), 2)]
+        srows = rows[:min(len(rows), 8)]                          # about 6 s of host work on 16 cores
         stoks = min(T, 4096)
         v, dt = oracle_prefill_sample(wl, inputs, srows, stoks, ncores)
         res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ncores, "kind": "oracle",
@@ -452,10 +456,10 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         ncores = len(os.sched_getaffinity(0))
-        stoks, ssteps = 2048, 32
-        v, dt = oracle_decode_sample(wl, inputs, rows[:1], stoks, ssteps, ncores)
+        stoks, ssteps = 2048, 256                                 # a few seconds of host work
+        v, dt = oracle_decode_sample(wl, inputs, rows[:4], stoks, ssteps, ncores)
         res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ncores, "kind": "oracle",
-                               "sample": f"batch row {rows[0]}, {ssteps} decode steps after a {stoks}-token prefill "
+                               "sample": f"batch rows {rows[:4]}, {ssteps} decode steps after a {stoks}-token prefill "
                                          f"(caches full; {dt:.1f} s timed)"}
     layer.close()
     return res
