@@ -297,15 +297,18 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
       }
       // weights 2^(z - m) <= 2^8 as bf16 pairs over the first half of this thread's S columns
-      float l0 = 0.f, l1 = 0.f;
+      // (packed f32x2 arithmetic: the sums of the even and of the odd columns are the two lanes)
+      const uint64_t sl22 = tc::pack_f2(sl2, sl2), nm2 = tc::pack_f2(-m_used, -m_used);
+      uint64_t lacc = tc::pack_f2(0.f, 0.f);
 #pragma unroll
       for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t pk[16];
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
-          const float p0 = tc::fast_exp2(fmaf(sv[c0 + j], sl2, -m_used)), p1 = tc::fast_exp2(fmaf(sv[c0 + j + 1], sl2, -m_used));
-          l0 += p0;
-          l1 += p1;
+          float x0, x1;
+          tc::unpack_f2(tc::fma2(tc::pack_f2(sv[c0 + j], sv[c0 + j + 1]), sl22, nm2), x0, x1);
+          const float p0 = tc::fast_exp2(x0), p1 = tc::fast_exp2(x1);
+          lacc = tc::add2(lacc, tc::pack_f2(p0, p1));
           pk[j >> 1] = pack_bf16x2(p0, p1);
         }
         asm volatile(
@@ -316,6 +319,8 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
             : "memory");
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      float l0, l1;
+      tc::unpack_f2(lacc, l0, l1);
       l += l0 + l1;
       tc::fence_before_sync();
       tc::mbar_arrive(BAR(A2_PREADY + w));

@@ -128,6 +128,9 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   const uint32_t tm_phi = tm_a + 192u;
   const uint32_t idesc1 = tc::make_idesc_bf16(128, 64, false, false);
   const uint32_t idesc2 = tc::make_idesc_bf16(128, d + 16, false, false);
+  // operand descriptors once; a K step adds its byte offset / 16 to the address field
+  const uint64_t dk = tc::make_desc_sw128(stage + S::st_k, 16, 1024), db1 = tc::make_desc_sw128(sbase + S::b1, 16, 1024),
+                 dht = tc::make_desc_sw128(sbase + S::ht, 16, 1024);
 
   if (wg == 1) asm volatile("bar.arrive 3, 512;" ::: "memory");   // row group 0 takes the first turn
 
@@ -150,8 +153,8 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     if (lead) {
 #pragma unroll
       for (int ks = 0; ks < d / 16; ++ks)
-        tc::mma_bf16_ss(tm_a, tc::make_desc_sw128(stage + S::st_k + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                        tc::make_desc_sw128(sbase + S::b1 + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), idesc1, ks > 0);
+        tc::mma_bf16_ss(tm_a, dk + (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                        db1 + (uint64_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), idesc1, ks > 0);
       tc::mma_commit(bar_mma);
     }
     ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
@@ -171,8 +174,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     if (lead) {
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ts(tm_a, tm_phi + ks * 8,
-                        tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024), idesc2, ks > 0);
+        tc::mma_bf16_ts(tm_a, tm_phi + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
       tc::mma_commit(bar_mma);
     }
     ok = tc::mbar_wait(bar_v, pv) && ok; pv ^= 1;
@@ -183,23 +185,30 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       tc::tmem_ld2(tm_a + lane_addr + d, dn);
       const float den = dn[0] + dn[1];
       const float inv = den > 0.f ? 1.0f / den : 0.f;
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      // packed pairs: d = v - P / den, four running sums of squares (columns 4k, 4k+1 | 4k+2, 4k+3)
+      const uint64_t ninv2 = tc::pack_f2(-inv, -inv);
+      uint64_t accA = tc::pack_f2(0.f, 0.f), accB = accA;
 #pragma unroll
       for (int c0 = 0; c0 < HC; c0 += 32) {
-        float p[32];
-        tc::tmem_ld32(tm_a + lane_addr + hf * HC + c0, p);
+        uint32_t p[32];
+        tc::tmem_ld32u(tm_a + lane_addr + hf * HC + c0, p);
 #pragma unroll
         for (int q8 = 0; q8 < 4; ++q8) {
           const int cc = hf * HC + c0 + q8 * 8;
-          uint4 raw = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (cc >> 6) * 16384 + tc::sw128_off(t, (cc & 63) >> 3));
-          float d0 = fmaf(p[q8 * 8 + 0], inv, -bf16lo_f(raw.x)), d1 = fmaf(p[q8 * 8 + 1], inv, -bf16hi_f(raw.x));
-          float d2 = fmaf(p[q8 * 8 + 2], inv, -bf16lo_f(raw.y)), d3 = fmaf(p[q8 * 8 + 3], inv, -bf16hi_f(raw.y));
-          float d4 = fmaf(p[q8 * 8 + 4], inv, -bf16lo_f(raw.z)), d5 = fmaf(p[q8 * 8 + 5], inv, -bf16hi_f(raw.z));
-          float d6 = fmaf(p[q8 * 8 + 6], inv, -bf16lo_f(raw.w)), d7 = fmaf(p[q8 * 8 + 7], inv, -bf16hi_f(raw.w));
-          a0 = fmaf(d0, d0, a0); a1 = fmaf(d1, d1, a1); a2 = fmaf(d2, d2, a2); a3 = fmaf(d3, d3, a3);
-          a0 = fmaf(d4, d4, a0); a1 = fmaf(d5, d5, a1); a2 = fmaf(d6, d6, a2); a3 = fmaf(d7, d7, a3);
+          const uint4 raw = *reinterpret_cast<const uint4*>(stage_p + S::st_v + (cc >> 6) * 16384 + tc::sw128_off(t, (cc & 63) >> 3));
+          const uint64_t d01 = tc::fma2(tc::pack_u2(p[q8 * 8 + 0], p[q8 * 8 + 1]), ninv2, tc::pack_u2(raw.x << 16, raw.x & 0xffff0000u));
+          const uint64_t d23 = tc::fma2(tc::pack_u2(p[q8 * 8 + 2], p[q8 * 8 + 3]), ninv2, tc::pack_u2(raw.y << 16, raw.y & 0xffff0000u));
+          const uint64_t d45 = tc::fma2(tc::pack_u2(p[q8 * 8 + 4], p[q8 * 8 + 5]), ninv2, tc::pack_u2(raw.z << 16, raw.z & 0xffff0000u));
+          const uint64_t d67 = tc::fma2(tc::pack_u2(p[q8 * 8 + 6], p[q8 * 8 + 7]), ninv2, tc::pack_u2(raw.w << 16, raw.w & 0xffff0000u));
+          accA = tc::fma2(d01, d01, accA);
+          accB = tc::fma2(d23, d23, accB);
+          accA = tc::fma2(d45, d45, accA);
+          accB = tc::fma2(d67, d67, accB);
         }
       }
+      float a0, a1, a2, a3;
+      tc::unpack_f2(accA, a0, a1);
+      tc::unpack_f2(accB, a2, a3);
       const float ss = (a0 + a1) + (a2 + a3);
       if (hf == 1) X.ssp[wg][t] = ss;
       tc::fence_async_smem();
