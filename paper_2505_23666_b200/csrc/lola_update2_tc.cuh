@@ -97,6 +97,20 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
         *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
     tc::grid_dep_wait();                             // the attention kernel has read the memories this kernel changes
   }
+  // everything the set-up needs from global memory is requested at once (one round trip): the work lists
+  // and their counts, the W^T image
+  int pre_cnt = 0, pre_fold = 0, pre_src = 0, pre_dst = 0;
+  uint4 pre_w[kblk];
+  if (PHASE == 2) {
+    pre_cnt = g_cnt[1];
+    if (tid < nF) pre_fold = g_fold[tid];
+    if (tid < min(L.cmax, kUp2MaxFold)) { pre_src = g_src[tid]; pre_dst = g_dst[tid]; }
+    if (fold) {
+      const uint4* img = wt_image + (size_t)h * kblk * 512;
+#pragma unroll
+      for (int q = 0; q < kblk; ++q) pre_w[q] = img[tid + q * kUp2Threads];
+    }
+  }
   // H of the unit streams into shared memory (asynchronous 16-byte copies) meanwhile
   if (PHASE != 1 && fold) {
     const float* Hg = L.H + (size_t)unit * D * d;
@@ -111,8 +125,13 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
     for (int i = tid; i < 4 * 256; i += kUp2Threads) (&X.hist[0][0])[i] = 0;
   // W^T image and zeroed operand tiles
   if (PHASE != 1 && fold) {
-    const uint4* img = wt_image + (size_t)h * kblk * 512;
-    for (int i = tid; i < kblk * 512; i += kUp2Threads) *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
+    if (PHASE == 2) {
+#pragma unroll
+      for (int q = 0; q < kblk; ++q) *reinterpret_cast<uint4*>(sm + S::b1 + (tid + q * kUp2Threads) * 16) = pre_w[q];
+    } else {
+      const uint4* img = wt_image + (size_t)h * kblk * 512;
+      for (int i = tid; i < kblk * 512; i += kUp2Threads) *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
+    }
     if (PHASE != 2)
       for (int i = tid; i < (32768 + 3 * 16384) / 16; i += kUp2Threads)
         *reinterpret_cast<uint4*>(sm + S::kt + i * 16) = make_uint4(0, 0, 0, 0);
@@ -253,10 +272,10 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
     return;
   }
   if (PHASE == 2) {
-    nMove = c.mode == UPD_NONE ? 0 : min(g_cnt[1], kUp2MaxFold);
+    nMove = c.mode == UPD_NONE ? 0 : min(pre_cnt, kUp2MaxFold);
     nGL = nMove;                                                     // every destination comes from the list
-    for (int i = tid; i < nF; i += kUp2Threads) X.fold_e[i] = g_fold[i];
-    for (int w = tid; w < nMove; w += kUp2Threads) { X.mover[w] = g_src[w]; X.free_slot[w] = g_dst[w]; }
+    if (tid < nF) X.fold_e[tid] = pre_fold;
+    if (tid < nMove) { X.mover[tid] = pre_src; X.free_slot[tid] = pre_dst; }
     __syncthreads();
   }
   // ---- leaving pairs that stay: into the freed slots, then into the slots beyond count_g
