@@ -186,6 +186,22 @@ int lola_prefill_chunk_host(lola_state* st, const void* q_host, const void* k_ho
 int lola_decode_step_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host,
                           void* out_host, void* staging_dev, size_t staging_bytes, void* stream);
 
+/* A run of `n_chunks` consecutive prefill chunks of `n_tokens` tokens each from HOST memory in one call
+ * (section "Chunkwise Inference": the chunks of a prompt in order).  q_host, k_host, v_host and out_host
+ * hold the chunks one after the other; chunk c is the tensor [B, n_tokens, heads, d] that
+ * lola_prefill_chunk takes, at byte offset c * (bytes of that tensor).  out_host (and then q_host) may be
+ * NULL: the memories are updated and no output is produced.
+ * `staging_dev`: device buffer of at least 2 * lola_staging_bytes(cfg, n_tokens) bytes (256-byte
+ * aligned): two sets of device copies, so that the copies in of chunk c + 1 and the copy out of chunk
+ * c - 1 run beside the kernels of chunk c.  The copies run on two streams that the handle creates at
+ * the first such call (host-side objects only; with them seven events); they start after the work
+ * already in `stream` and `stream` waits for them at the end.  The call returns after everything is
+ * complete: out_host is valid.  Host arrays should be pinned; pageable memory is correct but the copies
+ * then do not overlap.  Errors: ARG, SHAPE (n_tokens outside [1, max_chunk], n_chunks < 1), ALIGN, SIZE,
+ * CUDA, and those of lola_prefill_chunk (the run stops at the first failing chunk).                */
+int lola_prefill_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host, int32_t n_chunks,
+                      int32_t n_tokens, void* out_host, void* staging_dev, size_t staging_bytes, void* stream);
+
 /* Copies the three memories to the host arrays of `view` and synchronises `stream`.  The paper has
  * no counterpart; this is how results are inspected and checkpointed.  Returns LOLA_ERR_DEVICE if
  * the sticky status word is non-zero (the arrays are still filled).                             */

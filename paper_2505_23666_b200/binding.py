@@ -59,6 +59,7 @@ def _load() -> C.CDLL:
         "lola_decode_step_static": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "lola_staging_bytes": (sz, [cfgp, i32]),
         "lola_prefill_chunk_host": (C.c_int, [vp, vp, vp, vp, i32, vp, vp, sz, vp]),
+        "lola_prefill_host": (C.c_int, [vp, vp, vp, vp, i32, i32, vp, vp, sz, vp]),
         "lola_decode_step_host": (C.c_int, [vp, vp, vp, vp, vp, vp, sz, vp]),
         "lola_read_state": (C.c_int, [vp, viewp, vp]),
         "lola_write_state": (C.c_int, [vp, viewp, vp]),
@@ -79,7 +80,7 @@ def _load() -> C.CDLL:
 
 _lib = _load()
 EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_decode_step", "lola_decode_step_static", "lola_staging_bytes",
-           "lola_prefill_chunk_host", "lola_decode_step_host", "lola_read_state", "lola_write_state",
+           "lola_prefill_chunk_host", "lola_decode_step_host", "lola_prefill_host", "lola_read_state", "lola_write_state",
            "lola_reset_state", "lola_profile_enable", "lola_profile_read", "lola_launch_count", "lola_tokens_seen", "lola_set_tokens_seen", "lola_destroy_state", "lola_strerror"]
 
 
@@ -122,6 +123,11 @@ def lola_decode_step_static(st: int, q: int, k: int, v: int, out: int, stream: i
 def lola_prefill_chunk_host(st, q_host, k_host, v_host, n_tokens, out_host, staging_dev, staging_bytes, stream) -> int:
     return _lib.lola_prefill_chunk_host(st, q_host or None, k_host, v_host, int(n_tokens), out_host or None,
                                         staging_dev, staging_bytes, stream)
+
+
+def lola_prefill_host(st, q_host, k_host, v_host, n_chunks, n_tokens, out_host, staging_dev, staging_bytes, stream) -> int:
+    return _lib.lola_prefill_host(st, q_host or None, k_host, v_host, int(n_chunks), int(n_tokens), out_host or None,
+                                  staging_dev, staging_bytes, stream)
 
 
 def lola_decode_step_host(st, q_host, k_host, v_host, out_host, staging_dev, staging_bytes, stream) -> int:
@@ -250,6 +256,18 @@ class LolaLayer:
         _check(lola_prefill_chunk_host(self.handle, q.data_ptr() if want_out else 0, k.data_ptr(), v.data_ptr(), n,
                                        out.data_ptr() if want_out else 0, stg.data_ptr(), stg.numel(), self._stream()),
                "lola_prefill_chunk_host")
+        return out
+
+    def prefill_host(self, q, k, v, out=None, want_out=True):
+        """q, k, v (and out): host tensors [n_chunks, B, n_tokens, heads, d], the chunks in order."""
+        nch, n = k.shape[0], k.shape[2]
+        need = 2 * lola_staging_bytes(self.cfg, n)
+        if self._staging is None or self._staging.numel() < need:
+            self._staging = torch.empty(need, dtype=torch.uint8, device=self.device)
+        stg = self._staging
+        _check(lola_prefill_host(self.handle, q.data_ptr() if want_out else 0, k.data_ptr(), v.data_ptr(), nch, n,
+                                 out.data_ptr() if want_out else 0, stg.data_ptr(), stg.numel(), self._stream()),
+               "lola_prefill_host")
         return out
 
     def decode_step_host(self, q, k, v, out):

@@ -173,6 +173,9 @@ struct lola_state {
   bool himg_valid = false;             // the bf16 operand image of H matches H
   cudaStream_t aux = nullptr;          // second stream: Eq. 10 scoring runs beside the attention kernel
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // lola_prefill_host: two copy streams and the events that order them against the kernels (made at first use)
+  cudaStream_t cp_in = nullptr, cp_out = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
   bool force_chain = false;            // set while lola_decode_step_static runs: kernel chain with work lists
   CUtensorMap tm_gk, tm_gv, tm_wk, tm_wv;
   bool profiling = false;
@@ -632,6 +635,71 @@ int lola_decode_step_host(lola_state* st, const void* q_host, const void* k_host
   return run_host(st, q_host, k_host, v_host, 1, out_host, staging_dev, staging_bytes, stream, true);
 }
 
+static bool ensure_copy_streams(lola_state* st) {
+  if (st->cp_in) return true;
+  cudaEvent_t* evs[7] = {&st->ev_start, &st->ev_in[0], &st->ev_in[1], &st->ev_done[0], &st->ev_done[1], &st->ev_out[0], &st->ev_out[1]};
+  bool ok = cudaStreamCreateWithFlags(&st->cp_in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&st->cp_out, cudaStreamNonBlocking) == cudaSuccess;
+  for (cudaEvent_t* e : evs) ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    for (cudaEvent_t* e : evs) if (*e) { cudaEventDestroy(*e); *e = nullptr; }
+    if (st->cp_in) { cudaStreamDestroy(st->cp_in); st->cp_in = nullptr; }
+    if (st->cp_out) { cudaStreamDestroy(st->cp_out); st->cp_out = nullptr; }
+  }
+  return ok;
+}
+
+int lola_prefill_host(lola_state* st, const void* q_host, const void* k_host, const void* v_host, int32_t n_chunks,
+                      int32_t n_tokens, void* out_host, void* staging_dev, size_t staging_bytes, void* stream) {
+  if (!st || !k_host || !v_host || !staging_dev) return LOLA_ERR_ARG;
+  if (out_host && !q_host) return LOLA_ERR_ARG;
+  if (n_chunks < 1 || n_tokens < 1 || n_tokens > st->cfg.max_chunk) return LOLA_ERR_SHAPE;
+  if (!aligned(staging_dev, kAlign)) return LOLA_ERR_ALIGN;
+  const size_t per = lola_staging_bytes(&st->cfg, n_tokens);
+  if (staging_bytes < 2 * per) return LOLA_ERR_SIZE;
+  if (!ensure_copy_streams(st)) return LOLA_ERR_CUDA;
+  const lola_config& c = st->cfg;
+  const size_t es = elem_size(c), d = c.head_dim, B = c.batch;
+  const size_t qbytes = B * n_tokens * c.n_q_heads * d * es, kbytes = B * n_tokens * c.n_kv_heads * d * es;
+  const size_t qb = align_up(qbytes), kb = align_up(kbytes);
+  cudaStream_t s = (cudaStream_t)stream;
+  bool ok = cudaEventRecord(st->ev_start, s) == cudaSuccess && cudaStreamWaitEvent(st->cp_in, st->ev_start, 0) == cudaSuccess;
+  int rc = LOLA_OK;
+  bool out_pending[2] = {false, false};
+  for (int i = 0; ok && rc == LOLA_OK && i < n_chunks; ++i) {
+    const int b = i & 1;
+    char* p = (char*)staging_dev + (size_t)b * per;
+    void *qd = p, *kd = p + qb, *vd = p + qb + kb, *od = p + qb + 2 * kb;
+    // copies in (copy stream): this set of device copies is free once the kernels of chunk i - 2 are done
+    if (i >= 2) ok = ok && cudaStreamWaitEvent(st->cp_in, st->ev_done[b], 0) == cudaSuccess;
+    if (out_host) ok = ok && cudaMemcpyAsync(qd, (const char*)q_host + (size_t)i * qbytes, qbytes, cudaMemcpyHostToDevice, st->cp_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(kd, (const char*)k_host + (size_t)i * kbytes, kbytes, cudaMemcpyHostToDevice, st->cp_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(vd, (const char*)v_host + (size_t)i * kbytes, kbytes, cudaMemcpyHostToDevice, st->cp_in) == cudaSuccess;
+    ok = ok && cudaEventRecord(st->ev_in[b], st->cp_in) == cudaSuccess;
+    // kernels (caller's stream): after the copies in, and after the copy out of chunk i - 2 has read `od`
+    ok = ok && cudaStreamWaitEvent(s, st->ev_in[b], 0) == cudaSuccess;
+    if (out_pending[b]) ok = ok && cudaStreamWaitEvent(s, st->ev_out[b], 0) == cudaSuccess;
+    if (!ok) break;
+    rc = lola_prefill_chunk(st, out_host ? qd : nullptr, kd, vd, n_tokens, out_host ? od : nullptr, stream);
+    if (rc != LOLA_OK) break;
+    ok = ok && cudaEventRecord(st->ev_done[b], s) == cudaSuccess;
+    // copy out (second copy stream)
+    if (out_host) {
+      ok = ok && cudaStreamWaitEvent(st->cp_out, st->ev_done[b], 0) == cudaSuccess;
+      ok = ok && cudaMemcpyAsync((char*)out_host + (size_t)i * qbytes, od, qbytes, cudaMemcpyDeviceToHost, st->cp_out) == cudaSuccess;
+      ok = ok && cudaEventRecord(st->ev_out[b], st->cp_out) == cudaSuccess;
+      out_pending[b] = ok;
+    }
+  }
+  // everything joins the caller's stream again
+  for (int b = 0; b < 2; ++b)
+    if (out_pending[b]) ok = cudaStreamWaitEvent(s, st->ev_out[b], 0) == cudaSuccess && ok;
+  const bool synced = cudaStreamSynchronize(st->cp_in) == cudaSuccess && cudaStreamSynchronize(st->cp_out) == cudaSuccess &&
+                      cudaStreamSynchronize(s) == cudaSuccess;
+  if (rc != LOLA_OK) return rc;
+  return ok && synced ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
 int lola_read_state(const lola_state* st, const lola_state_view* view, void* stream) {
   if (!st || !view) return LOLA_ERR_ARG;
   const lola_config& c = st->cfg;
@@ -767,6 +835,10 @@ int lola_destroy_state(lola_state* st) {
   if (st->aux) { cudaStreamSynchronize(st->aux); cudaStreamDestroy(st->aux); }
   if (st->ev_fork) cudaEventDestroy(st->ev_fork);
   if (st->ev_join) cudaEventDestroy(st->ev_join);
+  if (st->cp_in) { cudaStreamSynchronize(st->cp_in); cudaStreamDestroy(st->cp_in); }
+  if (st->cp_out) { cudaStreamSynchronize(st->cp_out); cudaStreamDestroy(st->cp_out); }
+  for (cudaEvent_t e : {st->ev_start, st->ev_in[0], st->ev_in[1], st->ev_done[0], st->ev_done[1], st->ev_out[0], st->ev_out[1]})
+    if (e) cudaEventDestroy(e);
   delete st;
   return LOLA_OK;
 }

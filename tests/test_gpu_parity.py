@@ -159,6 +159,37 @@ def test_state_only_prefill_and_host_entry_points():
     b._cmp_out(out.float().numpy(), b.oracle.decode_step(q, k, v), "host decode")
 
 
+def test_prefill_host_run_of_chunks():
+    """lola_prefill_host (a run of chunks from pinned host memory, copies beside the kernels) gives the
+    same outputs and memories, bit for bit, as one lola_prefill_chunk call per chunk on device tensors."""
+    wl = small_case("hostrun", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=448, chunk=64,
+                    window=64, sparse=128, dtype="bf16", seed=23)
+    nch = wl.tokens // wl.chunk
+    a, b = Lockstep(wl, threads=1), Lockstep(wl, threads=1)
+    q, k, v = a.inputs.prefill_tokens(0, wl.tokens)
+
+    def chunks(x):                                   # [B, T, heads, d] -> [nch, B, C, heads, d]
+        t = torch.from_numpy(x).to(torch.bfloat16)
+        return t.reshape(t.shape[0], nch, wl.chunk, t.shape[2], t.shape[3]).permute(1, 0, 2, 3, 4).contiguous()
+
+    hq, hk, hv = (chunks(x).pin_memory() for x in (q, k, v))
+    hout = torch.empty_like(hq).pin_memory()
+    a.layer.prefill_host(hq, hk, hv, hout)
+    dq, dk, dv = (x.to(b.layer.device) for x in (hq, hk, hv))
+    for c in range(nch):
+        out = b.layer.prefill_chunk(dq[c], dk[c], dv[c])
+        assert torch.equal(out.cpu(), hout[c]), f"chunk {c}"
+    sa, sb = a.layer.read_state(), b.layer.read_state()
+    for key in ("H", "s", "sparse_pos", "sparse_k", "sparse_v", "window_k", "window_v"):
+        assert np.array_equal(sa[key], sb[key]), key
+    # and a state-only run (no outputs) leaves the same memories
+    c2 = Lockstep(wl, threads=1)
+    c2.layer.prefill_host(hq, hk, hv, want_out=False)
+    sc = c2.layer.read_state()
+    for key in ("H", "s", "sparse_pos", "sparse_k", "window_k"):
+        assert np.array_equal(sa[key], sc[key]), key
+
+
 def test_write_state_round_trip():
     wl = small_case("rt", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
                     dtype="f32", seed=9, scale_a=0.125)
