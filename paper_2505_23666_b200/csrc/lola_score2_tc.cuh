@@ -226,6 +226,10 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   if (warp == 0) tc::tmem_dealloc(tmem, 512);
   // ---- the last block of a unit to finish selects the pairs to fold (Eq. 12) from all the unit's scores
   __shared__ int is_last;
+  if (gridDim.x == 1) {                              // one block per unit: it has all the unit's scores
+    update2_body<DPL, 1>(L, c, wt_image, nullptr, sm, unit);
+    return;
+  }
   if (tid == 0) {
     int* arrived = L.counts + (size_t)unit * 4 + 2;
     const int prev = atomicAdd(arrived, 1);
