@@ -236,14 +236,14 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
   dim3 grid((L.g * c.nq + kAttRows - 1) / kAttRows, L.B * L.Hkv);
   if (st->have_maps && !st->force_chain && c.att_chunk == c.nq && c.nq <= 64 && c.n == c.nq) {
     // prefill chunk: TMA-fed, warp-specialised kernel; the call's q, k, v get their own descriptors
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, tout;
     if (make_tokens_map(&tq, c.q, L.B, c.nq, L.Hq, L.d) && make_tokens_map(&tk, c.k, L.B, c.n, L.Hkv, L.d) &&
-        make_tokens_map(&tv, c.v, L.B, c.n, L.Hkv, L.d)) {
+        make_tokens_map(&tv, c.v, L.B, c.n, L.Hkv, L.d) && make_tokens_map(&tout, c.out, L.B, c.nq, L.Hq, L.d)) {
       if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
       LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
       dim3 grid2(((L.g + 1) / 2 + 1) / 2, L.B * L.Hkv);
       const cudaError_t le = launch_pdl(k_attend2_tc<DPL>, grid2, dim3(kAt2Threads), Attend2Smem<DPL>::bytes, s, L, c, st->tm_gk, st->tm_gv,
-                                        st->tm_wk, st->tm_wv, tq, tk, tv, (const uint4*)(st->base + st->lay.wt),
+                                        st->tm_wk, st->tm_wv, tq, tk, tv, tout, (const uint4*)(st->base + st->lay.wt),
                                         (const __nv_bfloat16*)(st->base + st->lay.himg));
       return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
     }

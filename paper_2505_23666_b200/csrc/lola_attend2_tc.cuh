@@ -58,7 +58,8 @@ __global__ void __launch_bounds__(kAt2Threads, 1)
 k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
              const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
              const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_ck,
-             const __grid_constant__ CUtensorMap tm_cv, const uint4* wt_image, const __nv_bfloat16* ht_image) {
+             const __grid_constant__ CUtensorMap tm_cv, const __grid_constant__ CUtensorMap tm_out, const uint4* wt_image,
+             const __nv_bfloat16* ht_image) {
   using S = Attend2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
@@ -387,23 +388,40 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     ok = WAIT(A2_ODONE + w, NT & 1) && ok;
     tc::fence_after_sync();
     {
+      // the tile's outputs are staged in the free value buffer of stage w in the layout of a TMA box
+      // ([head slot][64-column block][64 tokens][128 bytes], 128-byte swizzle) and stored by one thread:
+      // 576 threads storing 16 bytes at a time would take the load/store unit 2 us
       const float inv = 1.0f / (X.hx[w][hf][t] + lden);
-      T* op = (T*)c.out + (((size_t)b * n + tok) * L.Hq + h * g + hl) * d + hf * HC;
+      uint8_t* stg = sm + S::stage0 + (size_t)w * S::stage_bytes + S::st_v;
+      const int hs = t >> 6;
 #pragma unroll
       for (int c0 = 0; c0 < HC; c0 += 32) {
         float ov[32];
         tc::tmem_ld32(tm_o + hf * HC + c0, ov);
-        if (row_ok && ok) {
 #pragma unroll
-          for (int q8 = 0; q8 < 4; ++q8) {
-            uint4 o;
-            o.x = pack_bf16x2(ov[q8 * 8 + 0] * inv, ov[q8 * 8 + 1] * inv);
-            o.y = pack_bf16x2(ov[q8 * 8 + 2] * inv, ov[q8 * 8 + 3] * inv);
-            o.z = pack_bf16x2(ov[q8 * 8 + 4] * inv, ov[q8 * 8 + 5] * inv);
-            o.w = pack_bf16x2(ov[q8 * 8 + 6] * inv, ov[q8 * 8 + 7] * inv);
-            *reinterpret_cast<uint4*>(op + c0 + q8 * 8) = o;
-          }
+        for (int q8 = 0; q8 < 4; ++q8) {
+          const int cc = hf * HC + c0 + q8 * 8;
+          uint4 o;
+          o.x = pack_bf16x2(ov[q8 * 8 + 0] * inv, ov[q8 * 8 + 1] * inv);
+          o.y = pack_bf16x2(ov[q8 * 8 + 2] * inv, ov[q8 * 8 + 3] * inv);
+          o.z = pack_bf16x2(ov[q8 * 8 + 4] * inv, ov[q8 * 8 + 5] * inv);
+          o.w = pack_bf16x2(ov[q8 * 8 + 6] * inv, ov[q8 * 8 + 7] * inv);
+          *reinterpret_cast<uint4*>(stg + (hs * kblk + (cc >> 6)) * 8192 + tc::sw128_off(tok, (cc & 63) >> 3)) = o;
         }
+      }
+      tc::fence_async_smem();
+      tc::named_bar_sync(1 + w, 256);
+      if (t == 0 && hf == 0 && ok) {
+        const uint32_t sstg = sbase + S::stage0 + (uint32_t)w * S::stage_bytes + S::st_v;
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const int hl2 = (qt0 + w) * 2 + s2;
+          if (hl2 >= g) continue;                      // (rows of tokens >= n lie outside the tensor: not written)
+#pragma unroll
+          for (int cb = 0; cb < kblk; ++cb)
+            tc::tma_store_4d(&tm_out, sstg + (uint32_t)(s2 * kblk + cb) * 8192u, cb * 64, h * g + hl2, 0, b);
+        }
+        tc::bulk_commit_group();
+        tc::bulk_wait_group_read();                    // the staging buffer stays valid until it is read
       }
     }
     if (!ok && t == 0 && hf == 0) atomicOr(L.status, 64);

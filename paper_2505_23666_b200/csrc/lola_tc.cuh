@@ -205,6 +205,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tmap,
       ::"r"(dst_smem), "l"((uint64_t)(uintptr_t)tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
+// One box of a rank-4 tensor map, shared -> global (bulk async-group completion).  Rows of the box that lie
+// outside the tensor are not written.  c0 as for the loads (16-byte aligned start); no negative coordinates.
+__device__ __forceinline__ void tma_store_4d(const void* tmap, uint32_t src_smem, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"((uint64_t)(uintptr_t)tmap),
+               "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src_smem)
+               : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)(uintptr_t)tmap) : "memory");
 }
@@ -224,6 +231,8 @@ __device__ __forceinline__ void bulk_reduce_add_f32(float* dst, uint32_t src_sme
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// (the copies have read their shared-memory source; their writes complete with the kernel at the latest)
+__device__ __forceinline__ void bulk_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // Programmatic dependent launch: a kernel launched with programmatic stream serialization may start
 // while the kernel before it in the stream still runs; it must pass grid_dep_wait() before it touches
 // anything that kernel (or an earlier one) produces or still reads.  Both are no-ops in a normal launch.
