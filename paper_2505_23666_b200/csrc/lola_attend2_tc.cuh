@@ -192,6 +192,8 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       tc::fence_after_sync();
       for (int w = 0; w < nw; ++w) issue_s(w, 0);
       tc::mma_commit(BAR(A2_KEMPTY + 0));
+      const int so = NT & 1;                                             // the W^T image sits in the key buffer of this stage
+      const uint32_t wt = sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k;
       for (int kt = 0; kt < NT; ++kt) {
         const int st = kt & 1;
         ok = WAIT(A2_VFULL + st, (kt >> 1) & 1) && ok;
@@ -200,29 +202,28 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
           ok = WAIT(A2_PREADY + w, kt & 1) && ok;
           tc::fence_after_sync();
           issue_pv(w, kt);
-          if (kt + 1 < NT) issue_s(w, kt + 1);
+          if (kt + 1 < NT) {
+            issue_s(w, kt + 1);
+          } else {
+            // after the last PV of this query tile, U = Q W of the linear term goes into its score columns
+            // (the tensor pipe runs in order: the weights there are consumed first)
+            if (w == 0) ok = WAIT(A2_WFULL, 0) && ok;
+#pragma unroll
+            for (int ks = 0; ks < d / 16; ++ks)
+              tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
+                              tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                              tc::make_desc_sw128(wt + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024),
+                              tc::make_idesc_bf16(128, 64, false, false), ks > 0);
+            tc::mma_commit(BAR(A2_SFULL + w));
+          }
         }
         tc::mma_commit(BAR(A2_VEMPTY + st));
         if (kt + 1 < NT) tc::mma_commit(BAR(A2_KEMPTY + (st ^ 1)));
       }
       // ---- linear term
-      const int so = NT & 1;
-      const uint32_t wt = sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k;
-      ok = WAIT(A2_WFULL, 0) && ok;
       ok = WAIT(A2_HFULL, 0) && ok;
       for (int w = 0; w < nw; ++w) {
-        ok = WAIT(A2_PREADY + w, NT & 1) && ok;                         // S_w free
-        tc::fence_after_sync();
-#pragma unroll
-        for (int ks = 0; ks < d / 16; ++ks)
-          tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
-                          tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                          tc::make_desc_sw128(wt + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024),
-                          tc::make_idesc_bf16(128, 64, false, false), ks > 0);
-        tc::mma_commit(BAR(A2_SFULL + w));
-      }
-      for (int w = 0; w < nw; ++w) {
-        ok = WAIT(A2_PREADY + w, (NT + 1) & 1) && ok;                   // scaled phi(Q_w) in tensor memory
+        ok = WAIT(A2_PREADY + w, NT & 1) && ok;                         // scaled phi(Q_w) in tensor memory
         tc::fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
@@ -327,10 +328,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       tc::mbar_arrive(BAR(A2_PREADY + w));
     }
     // ---- linear term: once the last PV of this tile has read P_w, S_w may be overwritten
-    ok = WAIT(A2_ODONE + w, (NT - 1) & 1) && ok;
-    tc::fence_after_sync();
-    tc::mbar_arrive(BAR(A2_PREADY + w));               // phase NT
-    ok = WAIT(A2_SFULL + w, NT & 1) && ok;
+    ok = WAIT(A2_SFULL + w, NT & 1) && ok;             // U = Q W is there (and every PV of this tile is complete)
     tc::fence_after_sync();
     float lden = 0.f;                                  // the other half of the row's denominator
     {
@@ -384,7 +382,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       lden = X.hx[w][hf ^ 1][t];
     }
     tc::fence_before_sync();
-    tc::mbar_arrive(BAR(A2_PREADY + w));               // phase NT + 1
+    tc::mbar_arrive(BAR(A2_PREADY + w));               // phase NT
     ok = WAIT(A2_ODONE + w, NT & 1) && ok;
     tc::fence_after_sync();
     {
