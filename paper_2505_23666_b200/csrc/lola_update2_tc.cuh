@@ -139,14 +139,21 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   int nGL = 0, nMove = 0;
   unsigned thr_key = 0;
   if (PHASE != 2) {
+  const unsigned key0 = __float_as_uint(scu[cg > 0 ? 0 : lam]);      // any one score: a guess at the leading byte
+  bool top_differs = false;
   for (int e = tid; e < nE; e += kUp2Threads) {
-    if (e < cg) { X.key[e] = __float_as_uint(scu[e]); X.pos[e] = L.gpos[(size_t)unit * lam + e]; }
-    else { X.key[e] = __float_as_uint(scu[lam + (e - cg)]); X.pos[e] = c.r_pos0 + (e - cg); }
+    unsigned k;
+    if (e < cg) { k = __float_as_uint(scu[e]); X.pos[e] = L.gpos[(size_t)unit * lam + e]; }
+    else { k = __float_as_uint(scu[lam + (e - cg)]); X.pos[e] = c.r_pos0 + (e - cg); }
+    X.key[e] = k;
+    top_differs = top_differs || ((k ^ key0) >> 24) != 0u;
   }
   // ---- 1. radix select of the nF lowest scores (scores are norms >= 0: bit patterns order like unsigned)
   unsigned prefix = 0, mask = 0, need = (unsigned)nF;
-  __syncthreads();
-  for (int pass = 0; pass < 4; ++pass) {
+  // scores of one unit are of one magnitude: when they all share the leading byte, its pass is skipped
+  const int first_pass = __syncthreads_or(top_differs ? 1 : 0) ? 0 : 1;
+  if (first_pass == 1) { prefix = key0 & 0xff000000u; mask = 0xff000000u; }
+  for (int pass = first_pass; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     for (int e = tid; e < nE; e += kUp2Threads) {
       const unsigned k = X.key[e];
