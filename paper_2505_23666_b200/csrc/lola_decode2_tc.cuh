@@ -2,10 +2,11 @@
 // a bf16 layer with F = 64, caches full, one pair leaving the window; at most 8 row tiles per unit).
 // Same arithmetic and the same per-tile products as k_decode_tc; what differs is who does what:
 //
-//   feature group (warps 0-7)   per tile: q.k columns and their row maxima, softmax weights (bf16) into
-//                               the Pr^T operand, the feature map of U into tensor memory
-//   score group   (warps 8-15)  per tile: Eq. 10 from [P | den] and the value tile, the tile's lowest
-//                               score, the row left out of O^T, the running sums of the weights
+//   feature group (warps 0-7)   per tile: q.k columns and their warp maxima into shared memory, the
+//                               feature map of U into tensor memory; no barrier inside the group
+//   score group   (warps 8-15)  per tile: running maxima and softmax weights (bf16) into the Pr^T operand,
+//                               Eq. 10 from [P | den] and the value tile, the tile's lowest score, the
+//                               row left out of O^T, the running sums of the weights
 //   warp 16, one thread         issues [U | Z] = K [W | Q^T] and [P | den] = phi [H | s]; key-tile loads
 //   warp 17, one thread         issues O^T += V^T Pr^T; value-tile loads
 //
@@ -31,13 +32,12 @@ struct Decode2Misc {
   uint4 new_kv[2 * 16];          // the new pair, bf16
   float zn[kDecQ], lden[kDecQ], dotL[kDecQ];
   float redmax[2][4][kDecQ];
-  float m_s[2][kDecQ];           // running maximum after tile t (log2 units)
+  float m_s[1][kDecQ];           // running maxima after the last tile (log2 units)
   float z_s[2][kDecQ][128];      // q.k of the tile's rows (log2 units)
   unsigned long long redkey[4];
   float red12[4][2];
   float ssp[128];                // partial squared errors of the second half of the value columns
   float l_s[4][kDecQ];
-  int moved[2][2];               // a running maximum grew in tile t (per half of the query rows)
   unsigned long long cand_key[kDec2MaxTiles];
   float cand_score[kDec2MaxTiles], cand_min2[kDec2MaxTiles];
   int cand_row[kDec2MaxTiles];
@@ -318,9 +318,6 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   } else if (role == 0) {
     // =================== feature group ===================
     // this thread's query rows: [hf * QH, hf * QH + QH)
-    float m_run[QH];
-#pragma unroll
-    for (int r = 0; r < QH; ++r) m_run[r] = 0.f;
     const bool exp_kind = L.phi_kind == 1;
     for (int tile = 0; tile < NT; ++tile) {
       const int i = tile & 1;
@@ -328,7 +325,8 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       const bool valid = R < lam || R - lam < eta;
       ok = tc::mbar_wait(bar_u(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
       tc::fence_after_sync();
-      float z[QH];
+      // q.k of this row (log2 units) and the warp's maxima: the score group turns them into weights
+      float z[QH], wm[QH];
       {
         float zraw[QH];
         if (QH == 4) tc::tmem_ld4(tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<float(&)[4]>(zraw));
@@ -336,8 +334,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
 #pragma unroll
         for (int r = 0; r < QH; ++r) {
           z[r] = valid ? zraw[r] * sl2 : -CUDART_INF_F;
-          float wm = warp_max_redux(z[r]);
-          if (lane == 0) X.redmax[i][wq][hf * QH + r] = wm;
+          wm[r] = warp_max_redux(z[r]);
         }
       }
       // this thread's half of the feature map: hf = 0: softmax(u), hf = 1: softmax(-u)
@@ -347,42 +344,19 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         tc::tmem_ld64u(tm_uz(i) + lane_addr, u);
         tc::phi_half(u, hf != 0, exp_kind, pk2);
       }
-      if (tile >= 2) {
-        // the buffers of tile - 2: its feature rows and q.k columns were used by the score group, its
-        // Pr^T operand by the O^T product
+      if (tile >= 2) {                               // the score group is done with the buffers of tile - 2
         ok = tc::mbar_wait(bar_ptready(i), (uint32_t)((tile - 2) >> 1) & 1u, abw) && ok;
-        const int ev = tile - 1;
-        ok = tc::mbar_wait(bar_o(ev & 1), (uint32_t)(ev >> 1) & 1u, abw) && ok;
         tc::fence_after_sync();
       }
       // bf16 pairs into tensor memory: the A operand of the second product (K index = feature j)
       tc::tmem_st32u(tm_phi(i) + lane_addr + hf * 32, pk2);
-      tc::named_bar_sync(1, 256);
-      // running maximum of q.k per query row (every valid row counts, also the one that will be folded:
-      // any m >= the true maximum leaves Eq. 14 unchanged), then the softmax weights of the tile (bf16;
-      // the sums use the rounded weights)
-      uint8_t* ptile = sm + stage_pt(i);
-      bool moved = false;
 #pragma unroll
       for (int r = 0; r < QH; ++r) {
-        const int rr = hf * QH + r;
-        const float m_new = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[i][0][rr], X.redmax[i][1][rr])),
-                                  fmaxf(X.redmax[i][2][rr], X.redmax[i][3][rr]));
-        moved = moved || (m_new != m_run[r]);
-        m_run[r] = m_new;
-        const float p = valid ? tc::fast_exp2(z[r] - m_new) : 0.f;
-        *reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2) =
-            (unsigned short)pack_bf16x2(p, 0.f);
-        X.z_s[i][rr][t] = z[r];
+        X.z_s[i][hf * QH + r][t] = z[r];
+        if (lane == 0) X.redmax[i][wq][hf * QH + r] = wm[r];
       }
-      if ((gtid & 127) == 0) {
-#pragma unroll
-        for (int r = 0; r < QH; ++r) X.m_s[i][hf * QH + r] = m_run[r];
-        X.moved[i][hf] = moved ? 1 : 0;
-      }
-      tc::fence_async_smem();
       tc::fence_before_sync();
-      tc::mbar_arrive(bar_phidone(i));
+      tc::mbar_arrive(bar_phidone(i));               // (release: the shared-memory writes above are visible to whoever acquires it)
     }
   } else {
     // =================== score group ===================
@@ -448,9 +422,11 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     tc::fence_async_smem();
     tc::mbar_arrive(bar_ht);
 
-    float lpart[QH], m_prev[QR];
+    // running maxima of q.k per query row (log2 units; every valid row counts, also the one that will be
+    // folded: any m >= the true maximum leaves Eq. 14 unchanged) and this thread's share of the sums
+    float lpart[QH], m_run[QR];
 #pragma unroll
-    for (int r = 0; r < QR; ++r) m_prev[r] = 0.f;
+    for (int r = 0; r < QR; ++r) m_run[r] = 0.f;
 #pragma unroll
     for (int r = 0; r < QH; ++r) lpart[r] = 0.f;
     for (int tile = 0; tile < NT; ++tile) {
@@ -464,8 +440,52 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       uint8_t* ptile = sm + stage_pt(i);
 
       ok = tc::mbar_wait(bar_vfull(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
-      ok = tc::mbar_wait(bar_p, (uint32_t)tile & 1u, abw) && ok;
+      ok = tc::mbar_wait(bar_p, (uint32_t)tile & 1u, abw) && ok;   // (its commit follows the feature group's arrival: z_s, redmax are visible)
+      if (tile >= 2) {                               // the Pr^T operand of tile - 2 was consumed by its O^T product
+        const int ev = tile - 1;
+        ok = tc::mbar_wait(bar_o(ev & 1), (uint32_t)(ev >> 1) & 1u, abw) && ok;
+      }
       tc::fence_after_sync();
+      // ---- softmax weights of the tile (bf16; the sums use the rounded weights) into the Pr^T operand
+      float pw[QH];
+      {
+        const bool valid = is_g || slot < eta;
+        float m_new[QR];
+        bool moved = false;
+#pragma unroll
+        for (int r = 0; r < QR; ++r) {
+          m_new[r] = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[i][0][r], X.redmax[i][1][r])),
+                           fmaxf(X.redmax[i][2][r], X.redmax[i][3][r]));
+          moved = moved || (m_new[r] != m_run[r]);
+        }
+        if (moved) {                                 // uniform over the group and rare after the first tiles
+          float alpha[QR];
+#pragma unroll
+          for (int r = 0; r < QR; ++r) alpha[r] = tc::fast_exp2(m_run[r] - m_new[r]);
+#pragma unroll
+          for (int r = 0; r < QH; ++r) lpart[r] *= hf ? alpha[QH + r] : alpha[r];
+          if (hf == 0) {
+            // O^T so far (the products up to the tile before, or the linear term) moves to the new maximum
+            ok = tc::mbar_wait(bar_o(tile & 1), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+            tc::fence_after_sync();
+            float ov[8];
+            tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+            for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
+            tc::tmem_st8(tm_o + lane_addr, ov);
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < QR; ++r) m_run[r] = m_new[r];
+#pragma unroll
+        for (int r = 0; r < QH; ++r) {
+          const int rr = hf * QH + r;
+          const float mr = hf ? m_run[QH + r] : m_run[r];
+          const uint32_t pb = pack_bf16x2(valid ? tc::fast_exp2(X.z_s[i][rr][t] - mr) : 0.f, 0.f);
+          pw[r] = bf16lo_f(pb);
+          *reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2) = (unsigned short)pb;
+        }
+      }
       // ---- Eq. 10: this thread's half of the value columns
       float score;
       {
@@ -561,34 +581,15 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
           for (int q = 0; q < 32; ++q) dst[q] = pr[q];
         }
       }
-      // sums of the weights the feature group wrote (the row left out gives its weights back)
-      if (X.moved[i][0] | X.moved[i][1]) {           // uniform over the block: some row's maximum grew
-        float alpha[QR];
-#pragma unroll
-        for (int r = 0; r < QR; ++r) {
-          const float mt = X.m_s[i][r];
-          alpha[r] = tc::fast_exp2(m_prev[r] - mt);
-          m_prev[r] = mt;
-        }
-#pragma unroll
-        for (int r = 0; r < QH; ++r) lpart[r] *= hf ? alpha[QH + r] : alpha[r];
-        if (hf == 0) {
-          // O^T so far (the products up to the tile before, or the linear term) moves to the new maximum
-          ok = tc::mbar_wait(bar_o(tile & 1), (uint32_t)(tile >> 1) & 1u, abw) && ok;
-          tc::fence_after_sync();
-          float ov[8];
-          tc::tmem_ld8(tm_o + lane_addr, ov);
-#pragma unroll
-          for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
-          tc::tmem_st8(tm_o + lane_addr, ov);
-        }
-      }
+      // sums of the weights (the row left out takes its weights back)
 #pragma unroll
       for (int r = 0; r < QH; ++r) {
-        const int rr = hf * QH + r;
-        unsigned short* wp = reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2);
-        if (left_out) *wp = 0;
-        else lpart[r] += __uint_as_float((uint32_t)(*wp) << 16);
+        if (left_out) {
+          const int rr = hf * QH + r;
+          *reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2) = 0;
+        } else {
+          lpart[r] += pw[r];
+        }
       }
       tc::fence_async_smem();
       tc::fence_before_sync();
@@ -598,6 +599,10 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     for (int r = 0; r < QH; ++r) {
       float ls = warp_sum(lpart[r]);
       if (lane == 0) X.l_s[wq][hf * QH + r] = ls;
+    }
+    if (gtid == 0) {
+#pragma unroll
+      for (int r = 0; r < QR; ++r) X.m_s[0][r] = m_run[r];
     }
   }
 
@@ -655,7 +660,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
 
   // ---- Eq. 14: thread (query row r, value column cc)
   if (okb) {
-    const int il = (NT - 1) & 1;
+    const int il = 0;                                // the score group left the final maxima there
     for (int i = tid; i < g * d; i += kDec2Threads) {
       const int r = i / d, cc = i % d;
       const float m0 = X.m_s[il][r];
