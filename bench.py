@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     "decode": {"sources": ["paper_2505_23666_b200/csrc/lola_decode2_tc.cuh", "paper_2505_23666_b200/csrc/lola_decode_tc.cuh",
                            "paper_2505_23666_b200/csrc/lola_tc.cuh"],
-               "sha256_16": "c728d724172c75bf", "bytes_per_launch": 304.2e6, "units": 512},
+               "sha256_16": "0f385b660aa94ed2", "bytes_per_launch": 303.8e6, "units": 512},
 }
 
 
