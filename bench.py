@@ -9,7 +9,10 @@ One "step" is one pass of the whole hot path over the workload's batch:
   * decode workload (cfg3): all `decode_steps` single-token lola_decode_step calls on a state built (untimed)
     by the seeded prefill; the state is restored from a device copy before every step.
 The printed value is tokens/s per layer (whole job, all GPUs).  The default line is the 8B-shaped prefill
-(cfg2) and carries the decode workload (cfg3) as a second entry under "decode".
+(cfg2) and carries the decode workload (cfg3) as a second entry under "decode" and the other three workloads
+(cfg0, cfg1, cfg4: tokens/s, per-chunk latency, fraction of the chip's peak and of the peak of the SMs they
+occupy, the oracle's tokens/s) under "workloads".  After every timed loop the state's status word is checked
+and, at one GPU, the outputs the loop left are compared with the CPU oracle's.
 
 Units are independent, so N GPUs each run the same per-GPU workload on their own batch rows (weak scaling,
 no data-path collective); torch.distributed is used only for the barrier and the max over ranks.
@@ -36,6 +39,8 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch from an ncu capture (profiles/), valid only
 # while the kernel's sources are the ones that were captured (first 16 hex digits of the SHA-256 over them)
 NCU_TRAFFIC = {
+    "attend": {"sources": ["paper_2505_23666_b200/csrc/lola_attend2_tc.cuh", "paper_2505_23666_b200/csrc/lola_tc.cuh"],
+               "sha256_16": "", "bytes_per_launch": 38.0e6, "units": 64},
     "decode": {"sources": ["paper_2505_23666_b200/csrc/lola_decode2_tc.cuh", "paper_2505_23666_b200/csrc/lola_decode_tc.cuh",
                            "paper_2505_23666_b200/csrc/lola_tc.cuh"],
                "sha256_16": "0f385b660aa94ed2", "bytes_per_launch": 303.8e6, "units": 512},
@@ -59,6 +64,10 @@ def ncu_traffic(kind, units):
     except OSError:
         return None
     return ent["bytes_per_launch"] * units / ent["units"]
+
+
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0,          # B200 data sheet: HBM3e (DGX figure) and dense bf16
+           "fp32_alu_tflops": 148 * 128 * 2 * 1.965e9 / 1e12}    # 148 SMs x 128 FMA lanes x 2 flop at 1965 MHz
 
 
 # ----------------------------------------------------------------------------- algorithmic work
@@ -189,30 +198,57 @@ def barrier(world: int):
         dist.barrier()
 
 
-def oracle_prefill_sample(wl, inputs, rows, tokens, threads):
-    """Times the CPU oracle as it stands on `rows` x `tokens` of the workload. Returns (tokens/s, seconds)."""
+def oracle_prefill_sample(wl, inputs, rows, tokens, threads, keep_last=False):
+    """Times the CPU oracle as it stands on `rows` x `tokens` of the workload.  Returns (tokens/s, seconds) and,
+    with keep_last, the oracle's outputs of the sample's last chunk."""
     from oracle.lola_oracle import LolaOracle, config_for
     orc = LolaOracle(config_for(wl, batch=len(rows)), inputs.W.astype(np.float64), threads=threads)
     chunks = [inputs.prefill_tokens(t, min(wl.chunk, tokens - t), batch_rows=rows) for t in range(0, tokens, wl.chunk)]
     t0 = time.time()
+    last = None
     for q, k, v in chunks:
-        orc.prefill_chunk(q, k, v)
+        last = orc.prefill_chunk(q, k, v)
     dt = time.time() - t0
-    return len(rows) * tokens / dt, dt
+    return (len(rows) * tokens / dt, dt, last) if keep_last else (len(rows) * tokens / dt, dt)
 
 
-def oracle_decode_sample(wl, inputs, rows, prefill_tokens, steps, threads):
+def oracle_decode_sample(wl, inputs, rows, prefill_tokens, steps, threads, keep=False):
+    """The oracle builds its own state from the seeded prefill (untimed), then `steps` generation steps are timed."""
     from oracle.lola_oracle import LolaOracle, config_for
     orc = LolaOracle(config_for(wl, batch=len(rows)), inputs.W.astype(np.float64), threads=threads)
     for t in range(0, prefill_tokens, wl.chunk):
         _, k, v = inputs.prefill_tokens(t, wl.chunk, batch_rows=rows, need_q=False)
         orc.prefill_chunk(None, k, v, want_out=False)
     toks = [inputs.decode_token(i, batch_rows=rows) for i in range(steps)]
+    outs = []
     t0 = time.time()
     for q, k, v in toks:
-        orc.decode_step(q, k, v)
+        outs.append(orc.decode_step(q, k, v))
     dt = time.time() - t0
-    return len(rows) * steps / dt, dt
+    return (len(rows) * steps / dt, dt, outs) if keep else (len(rows) * steps / dt, dt)
+
+
+def check_status(layer, where):
+    """The timed kernels skip their work once the state's status word is set: a timed loop only counts if the word
+    is still zero afterwards."""
+    st = layer.read_state(fields=("status",), check=False)
+    code = int(st["status"][0])
+    assert code == 0, f"{where}: device status word {code} after the timed loop - the timing is void"
+    return code
+
+
+def compare_units(got, ref, group, tol):
+    """got, ref [rows, ..., Hq, d]: per (row, KV head) unit the largest |got - ref|; returns the check record."""
+    import numpy as _np
+    got = _np.asarray(got, dtype=_np.float64)
+    ref = _np.asarray(ref, dtype=_np.float64)
+    assert _np.isfinite(got).all(), "non-finite output after the timed loop"
+    err = _np.abs(got - ref)
+    err = err.reshape(err.shape[:-2] + (err.shape[-2] // group, group, err.shape[-1]))
+    axes = tuple(i for i in range(err.ndim) if i not in (0, err.ndim - 3))
+    per_unit = err.max(axis=axes)                                   # [rows, Hkv]
+    return {"units": int(per_unit.size), "units_within_tol": int((per_unit <= tol).sum()), "tol": tol,
+            "worst_abs_err": float(per_unit.max())}
 
 
 # ----------------------------------------------------------------------------- prefill workloads
@@ -272,6 +308,8 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
     ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     launches = layer.launches - l0
     clocks = sampler.summary(w0, w1)
+    check_status(layer, f"{wl.name} prefill")
+    call_info = layer.last_call_info()                            # the last chunk call (caches full)
 
     # end to end through the host-buffer entry point (copies inside the timed region)
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -300,8 +338,16 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
     dom = max(kms, key=kms.get)
     dom_launch_ms = kms[dom] / kn[dom]
     dom_flops_per_launch = flops[dom] * prof_steps / kn[dom]
-    peak = peaks["bf16_tflops_sustained"]
+    # the burst figure bounds a timed region of well under a second at full clocks, the sustained one a long region
+    burst = ms * 1e-3 < 1.0
+    tensor = wl.dtype == "bf16"
+    peak = (peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]) if tensor else NOMINAL["fp32_alu_tflops"]
+    peak_src = (peaks["source"] + (" (burst bf16)" if burst else " (sustained bf16)")) if tensor else \
+        "derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1965 MHz"
     achieved = dom_flops_per_launch / (dom_launch_ms * 1e-3) / 1e12
+    whole = total_flops / (ms / args.steps * 1e-3) / 1e12
+    # thread blocks that run side by side in a call with full caches: attention and scoring
+    sms = min(148, call_info["ctas"].get("attend", 0) + call_info["ctas"].get("score", 0)) or 148
     tokens_per_step = B * T
     res = {
         "metric": METRIC, "value": world * tokens_per_step * args.steps / (ms * 1e-3), "unit": UNIT,
@@ -317,21 +363,34 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
                 "h2d_bytes_per_step": (hq.numel() + 2 * hk.numel()) * hq.element_size(),
                 "d2h_bytes_per_step": hout.numel() * hout.element_size(), "steps": e2e_steps},
         "gpu_launches": launches,
-        "roofline": {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
-                     "launch_us": dom_launch_ms * 1e3,
-                     "whole_step": {"achieved": total_flops / (ms / args.steps * 1e-3) / 1e12,
-                                    "frac": total_flops / (ms / args.steps * 1e-3) / 1e12 / peak},
+        "roofline": {"bound": "tensor" if tensor else "alu", "kernel": dom, "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": ncu_traffic(dom, wl.units) if "attend_tma" in call_info["paths"] else None,
+                     "peak_source": peak_src, "launch_us": dom_launch_ms * 1e3,
+                     "frac_nominal": achieved / (NOMINAL["bf16_tflops"] if tensor else NOMINAL["fp32_alu_tflops"]),
+                     "whole_step": {"achieved": whole, "frac": whole / peak,
+                                    "frac_nominal": whole / (NOMINAL["bf16_tflops"] if tensor else NOMINAL["fp32_alu_tflops"]),
+                                    "sms_occupied": sms, "frac_of_occupied_sms": whole / (peak * sms / 148.0)},
                      "kernel_ms_per_step": {k: v / prof_steps for k, v in kms.items()},
-                     "kernel_launches_per_step": {k: v / prof_steps for k, v in kn.items()}},
+                     "kernel_launches_per_step": {k: v / prof_steps for k, v in kn.items()},
+                     "kernel_paths": call_info["paths"]},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         ncores = len(os.sched_getaffinity(0))
         srows = rows[:min(len(rows), 8)]                          # about 6 s of host work on 16 cores
         stoks = min(T, 4096)
-        v, dt = oracle_prefill_sample(wl, inputs, srows, stoks, ncores)
+        v, dt, last = oracle_prefill_sample(wl, inputs, srows, stoks, ncores, keep_last=True)
         res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ncores, "kind": "oracle",
                                "sample": f"batch rows {srows}, first {stoks} tokens ({dt:.1f} s)"}
+        # the outputs the timed loop left for the sample's last chunk against the oracle's
+        ci = stoks // C - 1
+        got = dout[ci][:len(srows)].float().cpu().numpy()
+        tol = 2e-2 if wl.dtype == "bf16" else 1e-4 * float(np.abs(last).max())
+        chk = compare_units(got, last, wl.group, tol)
+        chk["what"] = f"outputs of chunk {ci} left by the timed loop vs the float64 oracle, batch rows {srows}"
+        chk["status"] = 0
+        res["check"] = chk
+        assert chk["units_within_tol"] >= 0.9 * chk["units"], f"timed outputs disagree with the oracle: {chk}"
     layer.close()
     return res
 
@@ -406,6 +465,9 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
     ms = max_over_ranks(total_ms, world, dev)
     launches = layer.launches - l0
     clocks = sampler.summary(w0, w1)
+    check_status(layer, f"{wl.name} decode")
+    call_info = layer.last_call_info()
+    timed_out = dout[:, 0].float().cpu().numpy()                  # outputs of this rank's first batch row, all steps
 
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     restore()
@@ -446,8 +508,11 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
                 "h2d_bytes_per_step": (hq.numel() + 2 * hk.numel()) * hq.element_size(),
                 "d2h_bytes_per_step": hout.numel() * hout.element_size(), "steps": e2e_steps},
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "+".join(sorted(kms)) + " (all kernels of one decode call)",
+        "roofline": {"bound": "hbm",
+                     "kernel": ("k_decode2_tc (the whole generation step is this one kernel)" if list(kms) == ["decode"]
+                                else "+".join(sorted(kms)) + " (all kernels of one decode call)"),
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_nominal": achieved / NOMINAL["hbm_gbs"], "kernel_paths": call_info["paths"],
                      "traffic": (ncu_traffic("decode", wl.units) if "decode" in kms and len(kms) == 1 else None),
                      "peak_source": peaks["source"], "bytes_per_call": step_bytes, "flops_per_call": step_flops,
                      "launch_us": kernel_ms_per_call * 1e3,
@@ -455,11 +520,17 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         ncores = len(os.sched_getaffinity(0))
-        stoks, ssteps = 2048, 256                                 # a few seconds of host work
-        v, dt = oracle_decode_sample(wl, inputs, rows[:4], stoks, ssteps, ncores)
+        ssteps = min(S, 64)                                       # the oracle builds its own state: the full prefill of one row
+        v, dt, outs = oracle_decode_sample(wl, inputs, rows[:1], T, ssteps, ncores, keep=True)
         res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ncores, "kind": "oracle",
-                               "sample": f"batch rows {rows[:4]}, {ssteps} decode steps after a {stoks}-token prefill "
-                                         f"(caches full; {dt:.1f} s timed)"}
+                               "sample": f"batch row {rows[0]}, {ssteps} decode steps ({dt:.1f} s timed) after its own "
+                                         f"{T}-token prefill (untimed)"}
+        chk = compare_units(timed_out[:ssteps][None], np.stack([o[0] for o in outs])[None], wl.group, 2e-2)
+        chk["what"] = (f"outputs of the first {ssteps} steps left by the timed loop vs the float64 oracle on its own "
+                       f"{T}-token state, batch row {rows[0]} (per unit: worst over the steps)")
+        chk["status"] = 0
+        res["check"] = chk
+        assert chk["units_within_tol"] >= 0.75 * chk["units"], f"timed outputs disagree with the oracle: {chk}"
     layer.close()
     return res
 
@@ -506,6 +577,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=0, help="decode calls per step of cfg3 (0 = the workload's 256)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="default line without the cfg3 entry")
+    ap.add_argument("--no-extra", action="store_true", help="default line without the cfg0, cfg1, cfg4 entries")
     args = ap.parse_args()
     from paper_2505_23666_b200.workloads import WORKLOADS
     rank, local_rank, world = dist_env()
@@ -542,8 +614,20 @@ def main():
         r3 = bench_decode(wl3, a3, rank, local_rank, world, peaks)
         res["decode"] = {k: r3[k] for k in ("value", "unit", "ms_per_step", "steps", "config", "e2e", "gpu_launches",
                                              "roofline", "clocks") if k in r3}
-        if "cpu_baseline" in r3:
-            res["decode"]["cpu_baseline"] = r3["cpu_baseline"]
+        for key in ("cpu_baseline", "check"):
+            if key in r3:
+                res["decode"][key] = r3[key]
+    if args.workload == "default" and not args.no_extra:
+        # the other three workloads, a few passes each (cfg4: 2048 dependent chunk calls per pass)
+        res["workloads"] = {}
+        for name, steps in (("cfg0", 10), ("cfg1", 10), ("cfg4", 2)):
+            ax = argparse.Namespace(**vars(args))
+            ax.steps = steps
+            ax.e2e_steps = 1
+            rx = bench_prefill(WORKLOADS[name], ax, rank, local_rank, world, peaks)
+            res["workloads"][name] = {k: rx[k] for k in ("value", "unit", "ms_per_step", "steps", "dtype", "config", "e2e",
+                                                         "gpu_launches", "roofline", "clocks", "cpu_baseline", "check")
+                                      if k in rx}
     if rank == 0:
         print(json.dumps(res), flush=True)
     if world > 1:

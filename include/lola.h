@@ -162,7 +162,8 @@ int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v
  * (3 * LOLA_STATIC_MAX_LIST_ENTRIES + 4 * LOLA_STATIC_MAX_UNITS) * 4 bytes = 832 KiB on every GPU
  * that loads the library, until the process exits.
  * Set-up: the first call on each device looks up the array's device address (a host-side query,
- * no allocation, with that device current); make that first call outside any stream capture.
+ * no allocation, with that device current; the look-up is serialised between host threads); make that
+ * first call outside any stream capture.
  * Sharing: all states and all calls on a device use the same array and it keeps the last call's
  * contents.  Nothing in it has to start at zero (each step writes every entry before reading it),
  * but two calls that overlap on the GPU (different streams, or different states on different
@@ -229,6 +230,49 @@ enum {
 };
 int lola_profile_enable(lola_state* st, int enable);
 int lola_profile_read(lola_state* st, double* ms_by_kind, int64_t* launches_by_kind, void* stream);
+
+/* What the last lola_prefill_chunk / lola_decode_step call of this handle enqueued (no counterpart in the
+ * paper).  Several kernel sets compute the same step: the TMA-fed tensor-core kernels serve bf16 layers with
+ * feat_half = 64, prefill chunks of at most 64 tokens and sparse caches filled in whole 64-slot blocks; other
+ * shapes run on first-generation tensor-core kernels or on shape-generic CUDA-core kernels, which are
+ * several times slower.  A caller that cares reads `paths` after a call (host-side; nothing is synchronised).
+ * `ctas[kind]` is the number of thread blocks launched per LOLA_KERNEL_* kind.                            */
+enum {
+  LOLA_PATH_ATTEND_TMA = 1u << 0,        /* Eq. 14 on the TMA-fed warp-specialised kernel                   */
+  LOLA_PATH_ATTEND_MMA = 1u << 1,        /* Eq. 14 on the first-generation tensor-core kernel               */
+  LOLA_PATH_ATTEND_GENERIC = 1u << 2,    /* Eq. 14 on CUDA cores                                            */
+  LOLA_PATH_SCORE_TMA = 1u << 3,         /* Eq. 10 (+ Eq. 12 in the same launch) on the TMA-fed kernel      */
+  LOLA_PATH_SCORE_MMA = 1u << 4,
+  LOLA_PATH_SCORE_GENERIC = 1u << 5,
+  LOLA_PATH_SELECT_KERNEL = 1u << 6,     /* Eq. 12 as a launch of its own                                   */
+  LOLA_PATH_APPLY_TMA = 1u << 7,         /* Eq. 13 fold on tensor cores, moves, window roll                 */
+  LOLA_PATH_UPDATE_GENERIC = 1u << 8,
+  LOLA_PATH_DECODE_FUSED = 1u << 9,      /* the generation step as one kernel (units of up to 8 row tiles)  */
+  LOLA_PATH_DECODE_FUSED_LONG = 1u << 10,/* the same for units of 9 to 16 row tiles                         */
+  LOLA_PATH_H_IMAGE_REBUILD = 1u << 11   /* the tensor-core operand image of H had to be rebuilt first      */
+};
+typedef struct lola_call_info {
+  uint32_t paths;                        /* OR of LOLA_PATH_*                                               */
+  int32_t launches;                      /* kernels enqueued by the call                                    */
+  int32_t ctas[LOLA_N_KERNEL_KINDS];
+} lola_call_info;
+int lola_last_call_info(const lola_state* st, lola_call_info* out);
+
+/* Bits of the sticky status word (lola_state_view.status).  Every wait inside a kernel is bounded; a wait
+ * that runs out, or an index outside its array, sets a bit, the kernel cleans up and returns, and every
+ * later kernel of the state returns at once, so the memories stay as they were when the failure happened.
+ * lola_read_state then returns LOLA_ERR_DEVICE; lola_reset_state or lola_write_state clear the word.     */
+enum {
+  LOLA_STATUS_LISTS = 1, LOLA_STATUS_SCORE_MMA = 2, LOLA_STATUS_ATTEND_MMA = 4, LOLA_STATUS_DECODE = 8,
+  LOLA_STATUS_SCORE = 16, LOLA_STATUS_APPLY = 32, LOLA_STATUS_ATTEND = 64, LOLA_STATUS_SELFTEST = 128,
+  LOLA_STATUS_PREFILL_RUN = 256
+};
+
+/* Failure-path self-test (no counterpart in the paper): enqueues one warp that waits, with the bounded wait
+ * every kernel uses, for a completion that never comes; after `limit_us` microseconds (1 .. 250000) the wait
+ * gives up and sets LOLA_STATUS_SELFTEST.  Nothing traps and nothing spins without limit; the context stays
+ * usable.  Afterwards the state behaves as after any device-side failure (see above).  Errors: ARG, CUDA. */
+int lola_selftest_wait_timeout(lola_state* st, int32_t limit_us, void* stream);
 
 /* Number of kernel launches this handle has enqueued so far. */
 int64_t lola_launch_count(const lola_state* st);

@@ -24,10 +24,12 @@ Readings taken where the paper is silent:
   * if phi(k)^T s is not > 0 (only when s = 0) the predicted value is 0;
   * the exponentials of Eq. 14 are evaluated as exp(z - m) with m = max(0, max z)
     applied to all three terms, which leaves the quotient unchanged;
-  * `operand_rounding="bf16"`: the bf16 mode of the library takes the selection
-    decision with phi(K_E) and H rounded to bf16 in the Eq. 10 contraction and
-    folds the rounded phi (Eq. 13); the oracle rounds the same operands so both
-    sides decide in the same precision.  Accumulation stays float64.
+  * `operand_rounding="none"` (the default everywhere) is the method in float64
+    on the inputs as given.  `operand_rounding="bf16"` is a diagnostic variant:
+    phi(K_E) and H are rounded to bf16 as operands of the Eq. 10 contraction,
+    which is what tensor-core operands of a bf16 library undergo; accumulation
+    stays float64 and Eq. 13 folds phi(k) itself.  Tests use it beside the default
+    to tell operand rounding apart from arithmetic mistakes.
 
 Parity pins: every function here is pinned by tests/test_oracle_pins.py
 (closed forms, brute force, library special cases).  The absolute values of
@@ -162,13 +164,14 @@ class UnitState:
             self.G_pos, self.G_k, self.G_v = E_pos, E_k, E_v
             self.G_score = np.concatenate([self.G_score, np.full(len(R_pos), np.nan)])
             return
-        f = self._rq(self._phi(E_k))                        # phi(K_E), rounded in bf16 mode
+        f = self._phi(E_k)                                  # phi(K_E)
         if lam == 0:                                        # no sparse cache: everything folds, no scoring
             keep = np.zeros((0,), dtype=np.int64)
             lose = np.arange(m)
             score = np.full(m, np.nan)
         else:
-            score = sre_scores(f, E_v, self._rq(self.H), self.s)    # state BEFORE this update's fold
+            # state BEFORE this update's fold; the "bf16" variant rounds the two operands of this contraction only
+            score = sre_scores(self._rq(f), E_v, self._rq(self.H), self.s)
             order = np.lexsort((E_pos, -score))             # score descending, then older first
             keep = np.sort(order[:lam])
             lose = np.sort(order[lam:])
@@ -344,9 +347,10 @@ class LolaOracle:
 
 
 def config_for(wl, **kw) -> OracleConfig:
-    """OracleConfig for a workload description (duck-typed: any object with the shape fields)."""
+    """OracleConfig for a workload description (duck-typed: any object with the shape fields).
+    The oracle is the method in float64 on the workload's (once-rounded) inputs; the operand roundings of
+    the library's bf16 mode are an option the caller asks for (`operand_rounding="bf16"`)."""
     base = dict(batch=wl.batch, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
-                feat_half=wl.feat_half, window=wl.window, sparse=wl.sparse,
-                operand_rounding=("bf16" if wl.dtype == "bf16" else "none"))
+                feat_half=wl.feat_half, window=wl.window, sparse=wl.sparse, operand_rounding="none")
     base.update(kw)
     return OracleConfig(**base)

@@ -38,6 +38,15 @@ class lola_state_view(C.Structure):
                  "window_count", "window_pos", "window_k", "window_v", "n_seen", "status")]
 
 
+class lola_call_info(C.Structure):
+    _fields_ = [("paths", C.c_uint32), ("launches", C.c_int32), ("ctas", C.c_int32 * 8)]
+
+
+PATH_BITS = ["attend_tma", "attend_mma", "attend_generic", "score_tma", "score_mma", "score_generic", "select_kernel",
+             "apply_tma", "update_generic", "decode_fused", "decode_fused_long", "h_image_rebuild"]
+LOLA_STATUS_SELFTEST = 128
+
+
 class LolaError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -66,6 +75,8 @@ def _load() -> C.CDLL:
         "lola_reset_state": (C.c_int, [vp, vp]),
         "lola_profile_enable": (C.c_int, [vp, C.c_int]),
         "lola_profile_read": (C.c_int, [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), vp]),
+        "lola_last_call_info": (C.c_int, [vp, C.POINTER(lola_call_info)]),
+        "lola_selftest_wait_timeout": (C.c_int, [vp, i32, vp]),
         "lola_launch_count": (i64, [vp]),
         "lola_tokens_seen": (i64, [vp]),
         "lola_set_tokens_seen": (C.c_int, [vp, i64]),
@@ -81,7 +92,8 @@ def _load() -> C.CDLL:
 _lib = _load()
 EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_decode_step", "lola_decode_step_static", "lola_staging_bytes",
            "lola_prefill_chunk_host", "lola_decode_step_host", "lola_prefill_host", "lola_read_state", "lola_write_state",
-           "lola_reset_state", "lola_profile_enable", "lola_profile_read", "lola_launch_count", "lola_tokens_seen", "lola_set_tokens_seen", "lola_destroy_state", "lola_strerror"]
+           "lola_reset_state", "lola_profile_enable", "lola_profile_read", "lola_last_call_info", "lola_selftest_wait_timeout",
+           "lola_launch_count", "lola_tokens_seen", "lola_set_tokens_seen", "lola_destroy_state", "lola_strerror"]
 
 
 # ---- one-to-one wrappers (pointers are integers: tensor.data_ptr(), stream.cuda_stream) ----
@@ -163,6 +175,20 @@ def lola_profile_read(st: int, stream: int):
     return ({k: ms[i] for i, k in enumerate(KERNEL_KINDS) if n[i]}, {k: n[i] for i, k in enumerate(KERNEL_KINDS) if n[i]})
 
 
+def lola_last_call_info(st: int) -> dict:
+    """{"paths": [names of the LOLA_PATH_* bits], "launches": n, "ctas": {kind: blocks}} of the last call."""
+    info = lola_call_info()
+    rc = _lib.lola_last_call_info(st, C.byref(info))
+    if rc != LOLA_OK:
+        raise LolaError(rc, "lola_last_call_info")
+    return {"paths": [n for i, n in enumerate(PATH_BITS) if info.paths >> i & 1], "launches": int(info.launches),
+            "ctas": {k: int(info.ctas[i]) for i, k in enumerate(KERNEL_KINDS) if info.ctas[i]}}
+
+
+def lola_selftest_wait_timeout(st: int, limit_us: int, stream: int) -> int:
+    return _lib.lola_selftest_wait_timeout(st, int(limit_us), stream)
+
+
 def lola_launch_count(st: int) -> int:
     return int(_lib.lola_launch_count(st))
 
@@ -181,11 +207,11 @@ def lola_destroy_state(st: int) -> int:
 
 # ---- convenience holder --------------------------------------------------------------------
 def make_config(batch, n_q_heads, n_kv_heads, head_dim, feat_half, window, sparse, max_chunk,
-                dtype="bf16", phi_kind="softmax", softmax_scale=0.0, generic_kernels=False) -> lola_config:
+                dtype="bf16", phi_kind="softmax", softmax_scale=0.0, generic_kernels=False, flags=0) -> lola_config:
     return lola_config(batch, n_q_heads, n_kv_heads, head_dim, feat_half, window, sparse, max_chunk,
                        LOLA_BF16 if dtype == "bf16" else LOLA_F32,
                        LOLA_PHI_EXP if phi_kind == "exp" else LOLA_PHI_SOFTMAX, float(softmax_scale),
-                       1 if generic_kernels else 0)
+                       int(flags) | (1 if generic_kernels else 0))
 
 
 def _check(rc: int, where: str):
@@ -341,6 +367,9 @@ class LolaLayer:
 
     def profile_read(self):
         return lola_profile_read(self.handle, self._stream())
+
+    def last_call_info(self) -> dict:
+        return lola_last_call_info(self.handle)
 
     @property
     def launches(self) -> int:

@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -178,6 +179,7 @@ struct lola_state {
   cudaEvent_t ev_start = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
   bool force_chain = false;            // set while lola_decode_step_static runs: kernel chain with work lists
   CUtensorMap tm_gk, tm_gv, tm_wk, tm_wv;
+  lola_call_info info = {};            // what the last prefill / decode call enqueued
   bool profiling = false;
   std::vector<ProfRecord> records;     // events in use since the last lola_profile_read
   std::vector<ProfRecord> pool;        // events ready for reuse
@@ -188,8 +190,11 @@ namespace {
 // Brackets one launch with a pair of events when profiling is on (kind = LOLA_KERNEL_*).
 struct LaunchScope {
   lola_state* st; cudaStream_t s; ProfRecord rec; bool on;
-  LaunchScope(lola_state* st_, int kind, cudaStream_t s_) : st(st_), s(s_), on(st_->profiling) {
+  LaunchScope(lola_state* st_, int kind, cudaStream_t s_, uint32_t path = 0, int ctas = 0) : st(st_), s(s_), on(st_->profiling) {
     st->launches++;
+    st->info.paths |= path;
+    st->info.launches++;
+    if (kind >= 0 && kind < LOLA_N_KERNEL_KINDS) st->info.ctas[kind] += ctas;
     if (!on) return;
     if (!st->pool.empty()) { rec = st->pool.back(); st->pool.pop_back(); }
     else if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) { on = false; return; }
@@ -223,7 +228,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 template <int DPL>
 int ensure_h_image(lola_state* st, cudaStream_t s) {
   if (st->himg_valid) return LOLA_OK;
-  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s, LOLA_PATH_H_IMAGE_REBUILD, st->L.B * st->L.Hkv);
   k_build_ht_image<DPL><<<st->L.B * st->L.Hkv, 256, 0, s>>>(st->L, (__nv_bfloat16*)(st->base + st->lay.himg));
   if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   st->himg_valid = true;
@@ -240,19 +245,20 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
     if (make_tokens_map(&tq, c.q, L.B, c.nq, L.Hq, L.d) && make_tokens_map(&tk, c.k, L.B, c.n, L.Hkv, L.d) &&
         make_tokens_map(&tv, c.v, L.B, c.n, L.Hkv, L.d) && make_tokens_map(&tout, c.out, L.B, c.nq, L.Hq, L.d)) {
       if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
-      LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
       dim3 grid2(((L.g + 1) / 2 + 1) / 2, L.B * L.Hkv);
+      LaunchScope scope(st, LOLA_KERNEL_ATTEND, s, LOLA_PATH_ATTEND_TMA, (int)(grid2.x * grid2.y));
       const cudaError_t le = launch_pdl(k_attend2_tc<DPL>, grid2, dim3(kAt2Threads), Attend2Smem<DPL>::bytes, s, L, c, st->tm_gk, st->tm_gv,
                                         st->tm_wk, st->tm_wv, tq, tk, tv, tout, (const uint4*)(st->base + st->lay.wt),
                                         (const __nv_bfloat16*)(st->base + st->lay.himg));
       return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
     }
   }
-  LaunchScope scope(st, LOLA_KERNEL_ATTEND, s);
   if (st->tensor_path && L.g * c.nq >= 64) {
     dim3 tgrid((L.g * c.nq + kAtM - 1) / kAtM, L.B * L.Hkv);
+    LaunchScope scope(st, LOLA_KERNEL_ATTEND, s, LOLA_PATH_ATTEND_MMA, (int)(tgrid.x * tgrid.y));
     k_attend_tc<DPL><<<tgrid, 128, AttendTcSmem<DPL>::bytes, s>>>(L, c);
   } else {
+    LaunchScope scope(st, LOLA_KERNEL_ATTEND, s, LOLA_PATH_ATTEND_GENERIC, (int)(grid.x * grid.y));
     k_attend<T, DPL><<<grid, 256, attend_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
   }
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
@@ -284,8 +290,8 @@ int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss, int busy
   const uint4* img = (const uint4*)(st->base + st->lay.wt);
   __nv_bfloat16* himg = (__nv_bfloat16*)(st->base + st->lay.himg);
   // the selection (Eq. 12) runs in the scoring kernel: the last block of a unit to finish does it
-  LaunchScope scope(st, LOLA_KERNEL_SCORE, ss);
   dim3 grid((NT + tpc - 1) / tpc, U);
+  LaunchScope scope(st, LOLA_KERNEL_SCORE, ss, LOLA_PATH_SCORE_TMA, (int)(grid.x * grid.y));
   k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
@@ -295,7 +301,7 @@ int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss, int busy
 template <int DPL>
 int launch_apply(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
-  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s, LOLA_PATH_APPLY_TMA, L.B * L.Hkv);
   const cudaError_t le = launch_pdl(k_update2_tc<DPL, 2>, dim3(L.B * L.Hkv), dim3(kUp2Threads), Update2Smem<DPL>::bytes, s, L, c,
                                     (const uint4*)(st->base + st->lay.wt), (__nv_bfloat16*)(st->base + st->lay.himg));
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
@@ -315,11 +321,12 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   if (c.mode == UPD_SELECT) {
     const int nE = c.count_g + c.r;
     dim3 grid((nE + kScoreRows - 1) / kScoreRows, U);
-    LaunchScope scope(st, LOLA_KERNEL_SCORE, s);
     if (st->tensor_path) {
       dim3 tgrid((nE + kScTile - 1) / kScTile, U);
+      LaunchScope scope(st, LOLA_KERNEL_SCORE, s, LOLA_PATH_SCORE_MMA, (int)(tgrid.x * tgrid.y));
       k_score_tc<DPL><<<tgrid, 128, ScoreTcSmem<DPL>::bytes, s>>>(L, c);
     } else {
+      LaunchScope scope(st, LOLA_KERNEL_SCORE, s, LOLA_PATH_SCORE_GENERIC, (int)(grid.x * grid.y));
       k_score<T, DPL><<<grid, 256, score_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
     }
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
@@ -327,13 +334,13 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   if (c.mode != UPD_NONE) {
     const int nE = c.count_g + c.r;
     size_t sm = (c.mode == UPD_SELECT) ? ((size_t)nE * 8 + (size_t)L.cmax * 4 + (size_t)nE + 16) : 0;
-    LaunchScope scope(st, LOLA_KERNEL_SELECT, s);
+    LaunchScope scope(st, LOLA_KERNEL_SELECT, s, LOLA_PATH_SELECT_KERNEL, U);
     k_select<<<U, 256, sm, s>>>(L, c);
     if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
   }
   if (st->have_maps && !st->force_chain && (c.mode == UPD_NONE || c.mode == UPD_APPEND) && c.r <= kUp2MaxFold)
     return launch_apply<DPL>(st, c, s);  // nothing folds: moves from the work lists and the window roll
-  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s);
+  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s, LOLA_PATH_UPDATE_GENERIC, U);
   if (c.mode == UPD_SELECT || c.mode == UPD_FOLD_ALL) st->himg_valid = false;   // H changes without its operand image
   k_update<T, DPL><<<U, kUpdThreads, update_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
@@ -367,8 +374,8 @@ int run_prefill(lola_state* st, Call c, cudaStream_t s) {
 template <int DPL>
 int launch_decode_fused(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
-  LaunchScope scope(st, LOLA_KERNEL_DECODE, s);
   const int n_tiles = (L.lam / 64 + (L.eta + 63) / 64 + 1) / 2;
+  LaunchScope scope(st, LOLA_KERNEL_DECODE, s, n_tiles <= kDec2MaxTiles ? LOLA_PATH_DECODE_FUSED : LOLA_PATH_DECODE_FUSED_LONG, L.B * L.Hkv);
   const uint4* wt = (const uint4*)(st->base + st->lay.wt);
   if (n_tiles <= kDec2MaxTiles) {          // the pipelined kernel; longer units run the two-row-group kernel
     if (L.g <= 4)
@@ -405,6 +412,23 @@ int run_decode(lola_state* st, Call c, cudaStream_t s) {
        : ((st)->cfg.head_dim == 128 ? fn<float, 4>(st, __VA_ARGS__) : fn<float, 2>(st, __VA_ARGS__)))
 
 size_t elem_size(const lola_config& c) { return c.dtype == LOLA_BF16 ? 2 : 4; }
+
+// One warp waits, with the same bounded wait every kernel uses, for an mbarrier phase that nothing
+// completes; the wait gives up after `limit_ns` and the failure is recorded like any other.
+__global__ void k_selftest_wait(int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  const uint32_t b = tc::smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    tc::mbar_init(b, 1);
+    tc::mbar_init_fence();
+  }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = tc::mbar_try_wait(b, 0) || tc::mbar_wait_slow(b, 0, &abort_word, limit_ns);
+  if (!ok) atomicOr(status, LOLA_STATUS_SELFTEST);
+}
 
 }  // namespace
 
@@ -565,6 +589,7 @@ int lola_prefill_chunk(lola_state* st, const void* q, const void* k, const void*
   if (st->n_seen + n_tokens > 0x7fffffffLL) return LOLA_ERR_SHAPE;
   if (!aligned(k, 16) || !aligned(v, 16) || (out && (!aligned(q, 16) || !aligned(out, 16)))) return LOLA_ERR_ALIGN;
   const Geometry g = plan(st->cfg, st->n_seen, n_tokens);
+  st->info = lola_call_info{};
   Call c{};
   c.q = q; c.k = k; c.v = v; c.out = out;
   c.n = n_tokens; c.nq = n_tokens; c.n_seen = (int)st->n_seen;
@@ -580,6 +605,7 @@ int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v
   if (st->n_seen + 1 > 0x7fffffffLL) return LOLA_ERR_SHAPE;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16)) return LOLA_ERR_ALIGN;
   const Geometry g = plan(st->cfg, st->n_seen, 1);
+  st->info = lola_call_info{};
   Call c{};
   c.q = q; c.k = k; c.v = v; c.out = out;
   c.n = 1; c.nq = 1; c.n_seen = (int)st->n_seen;
@@ -790,6 +816,7 @@ int lola_write_state(lola_state* st, const lola_state_view* v, void* stream) {
   ok = ok && h2d(L.wk, wk.data(), wk.size());
   ok = ok && h2d(L.wv, wv.data(), wv.size());
   if (v->threshold) ok = ok && h2d(L.thr, v->threshold, U * 2 * 4);
+  ok = ok && cudaMemsetAsync(L.status, 0, 4, s) == cudaSuccess;      // a replaced state starts healthy
   if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return LOLA_ERR_CUDA;   // host staging dies here
   st->n_seen = n_seen;
   st->himg_valid = false;
@@ -828,6 +855,20 @@ int lola_set_tokens_seen(lola_state* st, int64_t n_seen) {
   return LOLA_OK;
 }
 
+int lola_last_call_info(const lola_state* st, lola_call_info* out) {
+  if (!st || !out) return LOLA_ERR_ARG;
+  *out = st->info;
+  return LOLA_OK;
+}
+
+int lola_selftest_wait_timeout(lola_state* st, int32_t limit_us, void* stream) {
+  if (!st) return LOLA_ERR_ARG;
+  if (limit_us < 1 || limit_us > 250000) return LOLA_ERR_ARG;
+  st->launches++;
+  k_selftest_wait<<<1, 32, 0, (cudaStream_t)stream>>>(st->L.status, (unsigned long long)limit_us * 1000ull);
+  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+}
+
 int lola_destroy_state(lola_state* st) {
   if (!st) return LOLA_ERR_ARG;
   for (auto* v : {&st->records, &st->pool})
@@ -854,6 +895,8 @@ static __device__ __align__(256) int g_static_lists[3 * LOLA_STATIC_MAX_LIST_ENT
 
 static int* static_lists_for_current_device(int* rc_out) {
   static int* ptrs[64] = {nullptr};
+  static std::mutex mu;                // first calls from several host threads look the address up one at a time
+  std::lock_guard<std::mutex> lock(mu);
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *rc_out = LOLA_ERR_CUDA; return nullptr; }
   if (!ptrs[dev]) {

@@ -76,7 +76,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   volatile int* abortw = &X.abort_word;
   auto WAIT = [&](int i, uint32_t parity) { return tc::mbar_wait(BAR(i), parity, abortw); };
 
-  if (*reinterpret_cast<volatile int*>(L.status) != 0) return;     // an earlier kernel failed: do nothing
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   if ((uint32_t)(sm - smem_raw) + S::total > S::bytes) {            // (cannot happen with a 1024-byte aligned window)
     if (threadIdx.x == 0) atomicOr(L.status, 64);
     return;

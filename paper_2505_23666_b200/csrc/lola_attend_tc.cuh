@@ -26,6 +26,7 @@ struct AttendTcSmem {
 
 template <int DPL>
 __global__ void __launch_bounds__(128) k_attend_tc(Layer L, Call c) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   using S = AttendTcSmem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int F = 64, D = 128;

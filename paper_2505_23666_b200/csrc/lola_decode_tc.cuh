@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(kDecThreads, 1)
 k_decode_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image) {
   using S = DecodeSmem<DPL>;
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
   constexpr int F = 64, D = 128;

@@ -184,6 +184,7 @@ __host__ __device__ constexpr size_t attend_smem_floats(int D) {
 
 template <typename T, int DPL>
 __global__ void __launch_bounds__(256) k_attend(Layer L, Call c) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
   extern __shared__ float sm[];
   float* qs = sm;                                   // [16][d]
@@ -317,6 +318,7 @@ __host__ __device__ constexpr size_t score_smem_floats(int D) {
 
 template <typename T, int DPL>
 __global__ void __launch_bounds__(256) k_score(Layer L, Call c) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
   constexpr int RPW = 4;
   extern __shared__ float sm[];
@@ -381,6 +383,7 @@ __device__ __forceinline__ bool better(float sa, int pa, float sb, int pb) {
 }
 
 __global__ void __launch_bounds__(256) k_select(Layer L, Call c) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   extern __shared__ float sm[];
   const int unit = blockIdx.x, tid = threadIdx.x;
   const int nE = c.count_g + c.r;
@@ -473,6 +476,7 @@ __device__ __forceinline__ void copy_row(T* dst, const T* src, int d, int lane) 
 
 template <typename T, int DPL>
 __global__ void __launch_bounds__(kUpdThreads) k_update(Layer L, Call c) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
   extern __shared__ float sm[];
   float* xs = sm;                                   // [16][d]
@@ -501,7 +505,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update(Layer L, Call c) {
         locate_eligible<T>(L, c, unit, b, h, e, kp, vp);
         for (int j = lane; j < d; j += 32) { xs[warp * d + j] = ldf<T>(kp + j); vs[warp * d + j] = ldf<T>(vp + j); }
         __syncwarp();
-        warp_phi<T>(xs + warp * d, Wh, d, L.F, L.phi_kind, rq, phis + (size_t)warp * D, lane);
+        warp_phi<T>(xs + warp * d, Wh, d, L.F, L.phi_kind, false, phis + (size_t)warp * D, lane);   // Eq. 13 folds phi(k) itself
       }
       __syncthreads();
       const int nb = min(kUpdFB, nf - f0);

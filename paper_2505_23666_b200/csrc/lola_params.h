@@ -35,6 +35,13 @@ struct Layer {          // fixed for the life of a state
   const void* W;        // [Hkv, d, F]
 };
 
+// Sticky device status word: once a kernel has recorded a failure (a bounded wait that ran out, a bounds
+// violation) every later kernel of the state returns at once, so the memories stay as the failure left them
+// until lola_reset_state / lola_write_state.
+#ifdef __CUDACC__
+__device__ __forceinline__ bool state_failed(const Layer& L) { return *reinterpret_cast<volatile const int*>(L.status) != 0; }
+#endif
+
 struct Call {           // one prefill chunk or decode step
   const void* q;        // [B, nq, Hq, d]
   const void* k;        // [B, n, Hkv, d] incoming pairs

@@ -49,6 +49,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image,
             const __nv_bfloat16* ht_image, int tiles_per_cta) {
   using S = Score2Smem<DPL>;
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
   constexpr int D = 128;

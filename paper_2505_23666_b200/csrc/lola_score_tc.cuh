@@ -60,6 +60,7 @@ __device__ __forceinline__ void phi_from_u64(const float (&u0)[32], const float 
 
 template <int DPL>
 __global__ void __launch_bounds__(128) k_score_tc(Layer L, Call c) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   using S = ScoreTcSmem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int F = 64, D = 128;

@@ -166,7 +166,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+constexpr unsigned long long kWaitLimitNs = 250000000ull;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word,
+                                            unsigned long long limit_ns = kWaitLimitNs) {
   unsigned long long deadline = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -174,7 +176,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
     if ((it & 255u) == 255u) {
       if (abort_word && *abort_word) return false;
       const unsigned long long now = global_ns();
-      if (deadline == 0) deadline = now + 250000000ull;
+      if (deadline == 0) deadline = now + limit_ns;
       else if (now > deadline) {
         if (abort_word) *abort_word = 1;
         return false;
@@ -387,6 +389,31 @@ __device__ __forceinline__ void phi_half(const uint32_t (&u)[64], bool neg, bool
     out[q] = *reinterpret_cast<uint32_t*>(&pr);
   }
 }
+// The same half of the feature map in two bf16 parts, hi = bf16(phi) and lo = bf16(phi - hi): hi + lo carries
+// 16 significant bits.  Eq. 13 folds phi(k) itself into the fp32 state, so the fold's tensor-core product
+// takes both parts (two K blocks of one product) where Eq. 10's takes hi alone.
+__device__ __forceinline__ void phi_half_split(const uint32_t (&u)[64], bool neg, bool exp_kind, uint32_t (&hi)[32], uint32_t (&lo)[32]) {
+  const float kL = neg ? -1.4426950408889634f : 1.4426950408889634f;
+  float x[64];
+  float mm = -3.0e38f;
+#pragma unroll
+  for (int i = 0; i < 64; ++i) { x[i] = __uint_as_float(u[i]) * kL; mm = fmaxf(mm, x[i]); }
+  if (exp_kind) mm = 0.f;
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < 64; ++i) { x[i] = fast_exp2(x[i] - mm); sum += x[i]; }
+  const float inv = exp_kind ? 1.0f : 1.0f / sum;
+#pragma unroll
+  for (int q = 0; q < 32; ++q) {
+    const float a = x[2 * q] * inv, b = x[2 * q + 1] * inv;
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
+    const float2 hf = __bfloat1622float2(h2);
+    __nv_bfloat162 l2 = __floats2bfloat162_rn(a - hf.x, b - hf.y);
+    hi[q] = *reinterpret_cast<uint32_t*>(&h2);
+    lo[q] = *reinterpret_cast<uint32_t*>(&l2);
+  }
+}
+
 template <bool NEG>
 __device__ __forceinline__ void phi_half_packed(const uint32_t (&u)[64], bool exp_kind, uint32_t (&out)[32]) {
   phi_half(u, NEG, exp_kind, out);

@@ -6,7 +6,10 @@
 //   3. the folded pairs are gathered into operand tiles, phi(K_S) is recomputed
 //      (tcgen05.mma K_S W, feature map with one thread pair per row, rounded to bf16) and
 //      [dH | ds] = phi(K_S)^T [V_S | 1]   (tcgen05.mma, M = 128 features, N = d + 16, K = folded pairs)
-//      is added to H, s; the new H is also written as the bf16 operand image the other kernels load;
+//      is added to H, s.  Eq. 13 folds phi(k) itself into the fp32 state: phi goes in as two bf16 parts
+//      (hi in operand rows 0..63, lo = phi - hi in rows 64..127, the value rows repeated), so the product
+//      carries 16 significant bits of phi at no extra instruction.  The new H is also written as the bf16
+//      operand image the other kernels load;
 //   4. leaving pairs that stay move into the freed slots; the incoming pairs enter the window ring.
 // Every wait on an mbarrier is bounded; a wait that runs out sets bit 32 of the status word.
 #pragma once
@@ -20,7 +23,7 @@ namespace lola {
 
 constexpr int kUp2Threads = 512;
 constexpr int kUp2MaxE = 4096;      // eligible pairs this kernel handles (scores and positions in shared memory)
-constexpr int kUp2MaxFold = 128;    // folded pairs per call (one operand tile)
+constexpr int kUp2MaxFold = 64;     // folded pairs per call (half an operand tile: the other half holds the low parts)
 
 template <int DPL>
 struct Update2Smem {
@@ -322,9 +325,13 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
     locate_eligible<T>(L, c, unit, b, h, e, kp, vp);
     const uint4 val = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
     *reinterpret_cast<uint4*>(sm + (isv ? S::vt : S::kt) + (ch >> 3) * 16384 + tc::sw128_off(row, ch & 7)) = val;
+    if (isv)                                                         // the value row again, for the low parts of phi
+      *reinterpret_cast<uint4*>(sm + S::vt + (ch >> 3) * 16384 + tc::sw128_off(row + 64, ch & 7)) = val;
   }
-  if (tid < nF)                                                      // the column of ones (block kblk, column 0)
+  if (tid < nF) {                                                    // the column of ones (block kblk, column 0)
     *reinterpret_cast<T*>(sm + S::vt + kblk * 16384 + tc::sw128_off(tid, 0)) = __float2bfloat16_rn(1.0f);
+    *reinterpret_cast<T*>(sm + S::vt + kblk * 16384 + tc::sw128_off(tid + 64, 0)) = __float2bfloat16_rn(1.0f);
+  }
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
@@ -348,14 +355,20 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   else { ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1; }
   tc::fence_after_sync();
   if (tid < 256) {                                                   // one thread pair per row: half of the feature map each
-    uint32_t u[64], pk2[32];
-    tc::tmem_ld64u(tm_u + lane_addr, u);
-    tc::phi_half(u, hf != 0, L.phi_kind == 1, pk2);
-    // phi tile over the key tile (consumed): row = folded pair, 64 features per 128-byte row and block
+    uint32_t u[64], hi[32], lo[32];
+    tc::tmem_ld64u(tm_u + lane_addr, u);                             // (warp-wide: every lane takes part)
+    if (t < 64) {
+      tc::phi_half_split(u, hf != 0, L.phi_kind == 1, hi, lo);
+      // phi tile over the key tile (consumed): row = folded pair (hi parts) and 64 + folded pair (lo parts),
+      // 64 features per 128-byte row and block
 #pragma unroll
-    for (int ch = 0; ch < 8; ++ch)
-      *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t, ch)) =
-          make_uint4(pk2[ch * 4], pk2[ch * 4 + 1], pk2[ch * 4 + 2], pk2[ch * 4 + 3]);
+      for (int ch = 0; ch < 8; ++ch) {
+        *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t, ch)) =
+            make_uint4(hi[ch * 4], hi[ch * 4 + 1], hi[ch * 4 + 2], hi[ch * 4 + 3]);
+        *reinterpret_cast<uint4*>(sm + S::kt + hf * 16384 + tc::sw128_off(t + 64, ch)) =
+            make_uint4(lo[ch * 4], lo[ch * 4 + 1], lo[ch * 4 + 2], lo[ch * 4 + 3]);
+      }
+    }
   }
   asm volatile("cp.async.wait_all;" ::: "memory");
   tc::fence_async_smem();
@@ -364,8 +377,10 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   tc::fence_after_sync();
   if (tid == 0) {
     // [dH | ds] = phi^T [V | 1]: A = phi tile read MN-major (M = feature), B = value tile MN-major
-    const int ksteps = (nF + 15) / 16;
-    for (int ks = 0; ks < ksteps; ++ks)
+    // K index = operand row: hi parts of the folded pairs, then (from row 64) their lo parts; rows of no
+    // pair hold the feature map of a zero key against a zero value row
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
       tc::mma_bf16_ss(tm_d, tc::make_desc_sw128(sbase + S::kt + ks * 2048, 16384, 1024),
                       tc::make_desc_sw128(sbase + S::vt + ks * 2048, 16384, 1024),
                       tc::make_idesc_bf16(128, d + 16, true, true), ks > 0);
@@ -433,6 +448,7 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
 
 template <int DPL, int PHASE>
 __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, const uint4* wt_image, __nv_bfloat16* ht_image) {
+  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   update2_body<DPL, PHASE>(L, c, wt_image, ht_image, sm, (int)blockIdx.x);

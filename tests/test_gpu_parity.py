@@ -4,7 +4,23 @@ import pytest
 import torch
 
 from paper_2505_23666_b200.workloads import WORKLOADS, WorkloadInputs, small_case
-from tests.parity import Lockstep
+from tests.parity import BF16_MODES, Lockstep, assert_near_tie, compare_unit
+
+
+def modes_for(dtype):
+    """bf16 cases run against both oracles (the method in float64, and its variant with the library's operand
+    roundings); fp32 cases have one oracle."""
+    return BF16_MODES if dtype == "bf16" else ("plain",)
+
+
+def resync_cap(summ, per=100, floor=2):
+    """Near-tie divergences allowed in a run: `floor`, or one per `per` scored unit-updates.  Against the plain
+    oracle the rounding of the Eq. 10 operands moves scores by about 1e-4 of their size, which swaps a pair at the
+    threshold in about one of 150 updates of 896 candidates (measured: 19 events in 3200 at the 8B shapes, 145 in
+    31872 on the decode workload's prefill); against the mirror oracle in about one of 1000 (5 in 3200, 10 in 16272)."""
+    if summ["oracle"] == "plain":
+        per = min(per, 50)
+    return max(floor, summ["scored_updates"] // per)
 
 pytestmark = pytest.mark.gpu
 
@@ -47,67 +63,92 @@ SMALL = [
 ]
 
 
-@pytest.mark.parametrize("name,d,F,eta,lam,C,tokens,decode,dtype", SMALL, ids=[s[0] for s in SMALL])
-def test_small_cases(name, d, F, eta, lam, C, tokens, decode, dtype):
+SMALL_MODES = [(s, m) for s in SMALL for m in modes_for(s[8])]
+
+
+@pytest.mark.parametrize("case,mode", SMALL_MODES, ids=[f"{s[0]}-{m}" for s, m in SMALL_MODES])
+def test_small_cases(case, mode):
+    name, d, F, eta, lam, C, tokens, decode, dtype = case
     wl = small_case(name, batch=2, n_q_heads=4, n_kv_heads=2, head_dim=d, feat_half=F, tokens=tokens, chunk=C,
                     window=eta, sparse=lam, dtype=dtype, seed=11, decode_steps=decode,
                     scale_a=(0.125 if dtype == "f32" else 1.0))
-    ls = Lockstep(wl, threads=1)
+    ls = Lockstep(wl, threads=1, oracle_mode=mode)
     summ = drive(ls, tokens, C, decode)
-    assert summ["resyncs"] <= max(1, summ["scored_updates"] // 50), summ
+    assert summ["resyncs"] <= resync_cap(summ, per=50, floor=2), summ
     if name == "f32_all_softmax":
         st = ls.layer.read_state()
         assert np.all(st["H"] == 0) and np.all(st["s"] == 0)
 
 
+@pytest.mark.parametrize("mode", BF16_MODES)
 @pytest.mark.parametrize("g,batch", [(1, 3), (4, 2), (8, 1)])
-def test_fused_decode_group_sizes(g, batch):
+def test_fused_decode_group_sizes(g, batch, mode):
     """Fused generation step for 1, 4 and 8 query heads per KV head, then many steps in a row."""
     wl = small_case(f"fused_g{g}", batch=batch, n_q_heads=2 * g, n_kv_heads=2, head_dim=128, feat_half=64, tokens=384,
                     chunk=64, window=64, sparse=128, dtype="bf16", seed=13, decode_steps=40)
-    ls = Lockstep(wl, threads=1)
+    ls = Lockstep(wl, threads=1, oracle_mode=mode)
     summ = drive(ls, 384, 64, 40)
-    assert summ["resyncs"] <= 2, summ
+    assert summ["resyncs"] <= resync_cap(summ), summ
 
 
-def test_fused_decode_long_unit():
+@pytest.mark.parametrize("mode", BF16_MODES)
+def test_fused_decode_long_unit(mode):
     """A unit of more than 8 row tiles (lambda + window > 1024) takes the two-row-group generation kernel."""
     wl = small_case("fused_long", batch=1, n_q_heads=4, n_kv_heads=2, head_dim=128, feat_half=64, tokens=1280,
                     chunk=64, window=64, sparse=1088, dtype="bf16", seed=19, decode_steps=12)
-    ls = Lockstep(wl, threads=1)
+    ls = Lockstep(wl, threads=1, oracle_mode=mode)
     t = 0
     while t < wl.tokens:
-        ls.prefill(t, wl.chunk, want_out=False, check_state=(t + wl.chunk >= wl.tokens))
+        ls.prefill(t, wl.chunk, want_out=False, check_state=("members" if t + wl.chunk < wl.tokens else True))
         t += wl.chunk
     for sidx in range(wl.decode_steps):
         ls.decode(sidx)
     summ = ls.summary()
-    assert summ["resyncs"] <= 2, summ
+    assert summ["resyncs"] <= resync_cap(summ), summ
 
 
-def test_cfg3_shape_decode_sample():
+@pytest.mark.parametrize("mode", BF16_MODES)
+def test_cfg3_shape_decode_sample(mode):
     """Two batch rows of the decode workload at its full shapes (lambda 832, window 64, 4 query heads per KV
     head, d 128) after a shortened prefill that fills both caches, 48 fused steps against the oracle."""
     wl = WORKLOADS["cfg3"].with_(batch=2, tokens=2048, decode_steps=48)
-    ls = Lockstep(wl)
+    ls = Lockstep(wl, oracle_mode=mode)
     t = 0
     while t < wl.tokens:
-        ls.prefill(t, wl.chunk, want_out=False, check_state=(t + wl.chunk >= wl.tokens))
+        ls.prefill(t, wl.chunk, want_out=False, check_state=("members" if t + wl.chunk < wl.tokens else True))
         t += wl.chunk
     for sidx in range(wl.decode_steps):
         ls.decode(sidx)
     summ = ls.summary()
     print("cfg3 sample", summ)
-    assert summ["resyncs"] <= 2, summ
+    assert summ["resyncs"] <= resync_cap(summ), summ
+
+
+def test_cfg3_full_state_64_units():
+    """The decode workload at its stated size on 8 of its 64 batch rows (64 units; the units of the method are
+    independent): both sides consume the full seeded 32768-token prefill (keys and values only; membership
+    compared after every chunk, every memory after the last), then all 256 generation steps are compared
+    output by output and memory by memory against the float64 oracle."""
+    wl = WORKLOADS["cfg3"].with_(batch=8)
+    ls = Lockstep(wl, threads=16)
+    nch = wl.tokens // wl.chunk
+    for c in range(nch):
+        ls.prefill(c * wl.chunk, wl.chunk, want_out=False, check_state=("members" if c + 1 < nch else True))
+    pre = ls.summary()
+    for sidx in range(wl.decode_steps):
+        ls.decode(sidx)
+    summ = ls.summary()
+    print("cfg3 full state, batch rows 0-7: after the prefill", pre, "after 256 steps", summ)
+    assert summ["resyncs"] <= resync_cap(summ), summ
 
 
 @pytest.mark.parametrize("scale", [0.7, 3.0])
-def test_large_logits_move_the_stabiliser(scale):
+def test_large_logits_move_the_stabiliser(scale):  # (mirror oracle: this case is about the softmax, not the selection)
     """A softmax scale far above 1/sqrt(d) makes q.k exceed the stabiliser by many powers of two inside
     a tile, so the attention kernels must rescale what they have accumulated (sums, weights, outputs)."""
     wl = small_case("hot", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=448, chunk=64,
                     window=64, sparse=192, dtype="bf16", seed=17, decode_steps=6)
-    ls = Lockstep(wl, threads=1, softmax_scale=scale)
+    ls = Lockstep(wl, threads=1, softmax_scale=scale, oracle_mode="mirror")
     summ = drive(ls, 448, 64, 6)
     assert summ["resyncs"] <= 2, summ
 
@@ -121,17 +162,22 @@ def test_bf16_generic_kernels_flag():
 
 
 def test_exp_feature_map():
+    """Eq. 6 as printed, [exp(xW), exp(-xW)], fp32 mode (CUDA-core kernels)."""
     wl = small_case("exp", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
                     dtype="f32", seed=5, decode_steps=8, scale_a=0.125)
-    from oracle.lola_oracle import config_for, LolaOracle
-    from paper_2505_23666_b200 import binding
-    ls = Lockstep(wl, threads=1)
-    # rebuild both sides with the Eq. 6 feature map
-    ls.ocfg = config_for(wl, phi_kind="exp")
-    ls.oracle = LolaOracle(ls.ocfg, ls.inputs.W.astype(np.float64))
-    ls.cfg = binding.make_config(1, 2, 2, 64, 64, 16, 24, 16, dtype="f32", phi_kind="exp")
-    ls.layer = binding.LolaLayer(ls.cfg, ls.inputs.W)
+    ls = Lockstep(wl, threads=1, phi_kind="exp")
     drive(ls, 160, 16, 8)
+
+
+@pytest.mark.parametrize("mode", BF16_MODES)
+def test_exp_feature_map_tensor_core_kernels(mode):
+    """Eq. 6 as printed on the tensor-core kernels (bf16, F = 64): prefill chunks with full caches, then fused
+    generation steps.  Inputs are scaled so that exp(+-xW) stays within a few units."""
+    wl = small_case("exp_tc", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=448, chunk=64,
+                    window=64, sparse=128, dtype="bf16", seed=29, decode_steps=10, scale_a=0.25)
+    ls = Lockstep(wl, threads=1, phi_kind="exp", oracle_mode=mode)
+    summ = drive(ls, 448, 64, 10)
+    assert summ["resyncs"] <= resync_cap(summ), summ
 
 
 def test_state_only_prefill_and_host_entry_points():
@@ -190,6 +236,76 @@ def test_prefill_host_run_of_chunks():
         assert np.array_equal(sa[key], sc[key]), key
 
 
+def test_back_to_back_chunks_at_cfg2_shapes():
+    """The call sequence the benchmark times: 30 chunks (16 of them with full caches) of the 8B-shaped prefill
+    workload (64 units) enqueued without any host synchronisation, so that the kernels of neighbouring calls
+    overlap the way they do in production.  Run twice: once bare, once with a device-side copy of the whole
+    state after every call.  Both runs must agree bit for bit; the copies are then read through the C ABI and
+    compared with the oracle chunk by chunk, as are the outputs of every chunk.  A unit whose selection
+    differs from the oracle's at a verified near-tie is left out from that chunk on."""
+    from paper_2505_23666_b200 import binding
+    from tests.parity import close, oracle_for, tolerances
+    nch = 30
+    wl = WORKLOADS["cfg2"].with_(tokens=nch * 64)
+    inp = WorkloadInputs(wl)
+    q, k, v = inp.prefill_tokens(0, wl.tokens)
+    cfg = binding.make_config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window, wl.sparse,
+                              wl.chunk, dtype=wl.dtype)
+
+    def chunks(x, dev):                              # [B, T, heads, d] -> [nch, B, C, heads, d]
+        t = torch.from_numpy(x).to(torch.bfloat16)
+        return t.reshape(t.shape[0], nch, wl.chunk, t.shape[2], t.shape[3]).permute(1, 0, 2, 3, 4).contiguous().to(dev)
+
+    bare = binding.LolaLayer(cfg, inp.W)
+    dq, dk, dv = (chunks(x, bare.device) for x in (q, k, v))
+    out_bare = torch.empty_like(dq)
+    for c in range(nch):
+        bare.prefill_chunk(dq[c], dk[c], dv[c], out=out_bare[c])
+    copied = binding.LolaLayer(cfg, inp.W)
+    out_copied = torch.empty_like(dq)
+    snaps = torch.empty((nch, copied.nbytes), dtype=torch.uint8, device=copied.device)
+    for c in range(nch):
+        copied.prefill_chunk(dq[c], dk[c], dv[c], out=out_copied[c])
+        snaps[c].copy_(copied.state)                 # stream-ordered device copy: no host synchronisation
+    torch.cuda.synchronize()
+    assert torch.equal(out_bare, out_copied)
+    sa, sb = bare.read_state(), copied.read_state()
+    for key in ("H", "s", "sparse_pos", "sparse_k", "sparse_v", "window_k", "window_v"):
+        assert np.array_equal(sa[key], sb[key]), key
+    # the oracle, chunk by chunk, against the outputs and the copied states
+    mode = "mirror"
+    tol = tolerances(wl.dtype, mode)
+    orc = oracle_for(wl, inp, wl.batch, mode, threads=16)
+    reader = binding.LolaLayer(cfg, inp.W)
+    worst = {"out": 0.0, "H": 0.0, "s": 0.0, "score": 0.0, "tie": 0.0}
+    gone = set()                                     # units that took the other side of a near-tie
+    g_ = wl.group
+    got = out_bare.float().cpu().numpy()
+    for c in range(nch):
+        ref = orc.prefill_chunk(q[:, c * 64:(c + 1) * 64], k[:, c * 64:(c + 1) * 64], v[:, c * 64:(c + 1) * 64])
+        for b in range(wl.batch):
+            for h in range(wl.n_kv_heads):
+                if (b, h) in gone:
+                    continue
+                ok, ratio = close(got[c, b, :, h * g_:(h + 1) * g_], ref[b, :, h * g_:(h + 1) * g_], tol["out"], tol["kind"])
+                worst["out"] = max(worst["out"], ratio)
+                assert ok, f"chunk {c} unit ({b},{h}): output outside tolerance ({ratio:.3g})"
+        reader.state.copy_(snaps[c])
+        binding.lola_set_tokens_seen(reader.handle, (c + 1) * 64)
+        gst = reader.read_state()
+        for b in range(wl.batch):
+            for h in range(wl.n_kv_heads):
+                if (b, h) in gone:
+                    continue
+                u = orc.units[b][h]
+                members = compare_unit(gst, u, b, h, tol, f"chunk {c}", worst)
+                if members is not None:
+                    assert_near_tie(u, members, tol["tie"], f"chunk {c}", (b, h), worst)
+                    gone.add((b, h))
+    print("back to back:", dict(worst=worst, units_left_out=sorted(gone)))
+    assert len(gone) <= 2, gone
+
+
 def test_write_state_round_trip():
     wl = small_case("rt", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
                     dtype="f32", seed=9, scale_a=0.125)
@@ -222,6 +338,40 @@ def test_argument_errors_leave_state_untouched():
     ls.prefill(0, 16)                                   # the state still works
 
 
+def test_bounded_wait_runs_out_and_is_reported():
+    """Failure path without a fault: a wait that nothing ends gives up after its limit (1 ms here) and sets
+    the sticky status word; the kernels of later calls return at once, so the memories stay as they were;
+    lola_read_state reports LOLA_ERR_DEVICE; lola_reset_state brings the state back."""
+    from paper_2505_23666_b200 import binding as b
+    wl = small_case("waits", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=448, chunk=64,
+                    window=64, sparse=128, dtype="bf16", seed=31, decode_steps=2)
+    ls = Lockstep(wl, threads=1, oracle_mode="mirror")
+    drive(ls, 384, 64)
+    L = ls.layer
+    before = L.read_state()
+    s = torch.cuda.current_stream().cuda_stream
+    assert b.lola_selftest_wait_timeout(L.handle, 0, s) == b.LOLA_ERR_ARG
+    assert b.lola_selftest_wait_timeout(None, 1000, s) == b.LOLA_ERR_ARG
+    assert b.lola_selftest_wait_timeout(L.handle, 1000, s) == b.LOLA_OK
+    q, k, v = ls.inputs.prefill_tokens(384, 64)
+    out = torch.full(q.shape, float("nan"), dtype=torch.bfloat16, device=L.device)
+    L.prefill_chunk(L.to_device(q), L.to_device(k), L.to_device(v), out=out)      # enqueues; its kernels do nothing
+    dq, dk, dv = (L.to_device(a) for a in ls.inputs.decode_token(0))
+    L.decode_step(dq, dk, dv)
+    with pytest.raises(b.LolaError) as ei:
+        L.read_state()
+    assert ei.value.code == b.LOLA_ERR_DEVICE
+    after = L.read_state(check=False)
+    assert int(after["status"][0]) == b.LOLA_STATUS_SELFTEST
+    assert torch.isnan(out.float()).all()
+    for key in ("H", "s", "sparse_pos", "sparse_k", "sparse_v", "window_k", "window_v"):
+        assert np.array_equal(before[key], after[key]), key
+    L.reset()
+    assert int(L.read_state()["status"][0]) == 0 and L.tokens_seen == 0
+    fresh = Lockstep(wl, threads=1, oracle_mode="mirror")                          # the context is still usable
+    drive(fresh, 128, 64)
+
+
 # ---- the five workloads
 def test_cfg0_full():
     wl = WORKLOADS["cfg0"]
@@ -231,27 +381,30 @@ def test_cfg0_full():
     assert summ["resyncs"] == 0 or summ["resyncs"] <= 1
 
 
-def test_cfg1_full():
+@pytest.mark.parametrize("mode", BF16_MODES)
+def test_cfg1_full(mode):
     wl = WORKLOADS["cfg1"]
-    ls = Lockstep(wl)
+    ls = Lockstep(wl, oracle_mode=mode)
     summ = drive(ls, wl.tokens, wl.chunk)
     print("cfg1", summ)
-    assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100)
+    assert summ["resyncs"] <= resync_cap(summ), summ
 
 
-def test_cfg2_full():
+@pytest.mark.parametrize("mode", BF16_MODES)
+def test_cfg2_full(mode):
     wl = WORKLOADS["cfg2"]
-    ls = Lockstep(wl)
+    ls = Lockstep(wl, threads=16, oracle_mode=mode)
     summ = drive(ls, wl.tokens, wl.chunk)
     print("cfg2", summ)
-    assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100)
+    assert summ["resyncs"] <= resync_cap(summ), summ
 
 
-def test_cfg4_needles_full_length():
+@pytest.mark.parametrize("mode", BF16_MODES)
+def test_cfg4_needles_full_length(mode):
     """The long-context workload at full size (131072 tokens, 8 units): outputs of every chunk against the
     oracle, the memories after every chunk, and the number of planted pairs that end in the sparse cache."""
     wl = WORKLOADS["cfg4"]
-    ls = Lockstep(wl, threads=8)
+    ls = Lockstep(wl, threads=8, oracle_mode=mode)
     nch = wl.tokens // wl.chunk
     for c in range(nch):
         ls.prefill(c * wl.chunk, wl.chunk)
@@ -263,4 +416,4 @@ def test_cfg4_needles_full_length():
     orc_count = ls.oracle.needle_count(ls.inputs.needle_pos)
     print("cfg4", summ, "needles in the sparse cache (oracle / library):", int(orc_count.sum()), int(gpu_count.sum()))
     assert np.array_equal(gpu_count, orc_count)
-    assert summ["resyncs"] <= max(2, summ["scored_updates"] // 100), summ
+    assert summ["resyncs"] <= resync_cap(summ), summ

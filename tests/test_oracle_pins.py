@@ -23,6 +23,15 @@ def lib_phi(x, W, kind="softmax"):
     return np.concatenate([scipy.special.softmax(u, axis=1), scipy.special.softmax(-u, axis=1)], axis=1)
 
 
+def nearest_bf16(x):
+    """Nearest value with 8 significant bits (ties to even) of float64 data, by scaling to integers: an
+    independent statement of the rounding (a cast through float32 would round twice)."""
+    x = np.asarray(x, dtype=np.float64)
+    e = np.floor(np.log2(np.abs(np.where(x == 0, 1.0, x))))
+    ulp = 2.0 ** (e - 7)
+    return np.where(x == 0, 0.0, np.rint(x / ulp) * ulp)
+
+
 def make_unit(d=8, F=4, eta=4, lam=3, kind="softmax", rounding="none", schedule="eager", rng=RNG):
     cfg = OracleConfig(1, 1, 1, d, F, eta, lam, phi_kind=kind, operand_rounding=rounding, schedule=schedule)
     W = rng.standard_normal((d, F)) / np.sqrt(d)
@@ -261,23 +270,18 @@ def test_conservation_and_selection(eta, lam, C, tail, rounding):
         for i, p in enumerate(u.G_pos):
             assert np.array_equal(u.G_k[i], k[p]) and np.array_equal(u.G_v[i], v[p])
         # H, s are the sum over folded pairs, from scratch
+        # (Eq. 13 folds phi(k) itself in both variants; the "bf16" variant rounds operands of Eq. 10 only)
         f = lib_phi(k[sorted(fold)], W) if fold else np.zeros((0, 2 * F))
-        if rounding == "bf16":
-            import torch
-            f = torch.tensor(f).to(torch.bfloat16).to(torch.float64).numpy()
         np.testing.assert_allclose(u.H, f.T @ v[sorted(fold)] if fold else 0 * u.H, rtol=1e-10, atol=1e-12)
         np.testing.assert_allclose(u.s, f.sum(0) if fold else 0 * u.s, rtol=1e-10, atol=1e-12)
-        if rounding == "none":
-            np.testing.assert_allclose(u.s.sum(), 2.0 * len(fold), rtol=1e-10)
+        np.testing.assert_allclose(u.s.sum(), 2.0 * len(fold), rtol=1e-10)
         # the selection equals a full sort of the eligible set scored against the state before the fold
         if newly and lam > 0:
             E = sorted(G | newly)
             fE = lib_phi(k[E], W)
             H0r = H0
             if rounding == "bf16":
-                import torch
-                fE = torch.tensor(fE).to(torch.bfloat16).to(torch.float64).numpy()
-                H0r = torch.tensor(H0).to(torch.bfloat16).to(torch.float64).numpy()
+                fE, H0r = nearest_bf16(fE), nearest_bf16(H0)
             den = fE @ s0
             vh = np.where(den[:, None] > 0, (fE @ H0r) / np.where(den > 0, den, 1.0)[:, None], 0.0)
             sc = np.linalg.norm(vh - v[E], axis=1)

@@ -25,6 +25,44 @@ def _prefilled(wl, inp):
     return layer
 
 
+def test_static_scratch_decode_matches_fused_decode():
+    """At shapes where lola_decode_step runs as the single fused kernel (bf16, lambda a multiple of 64) the
+    static variant runs the kernel chain instead: same step, other kernels, so outputs agree to the bf16
+    tolerance, not bit for bit.  A unit where the two resolved a tie at the selection threshold differently
+    (the reference's lowest kept and highest folded scores within 1e-4 of each other) is left out."""
+    wl = small_case("noalloc128", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=384, chunk=64,
+                    window=64, sparse=128, dtype="bf16", seed=22)
+    inp = WorkloadInputs(wl)
+    ref, new = _prefilled(wl, inp), _prefilled(wl, inp)
+    s = torch.cuda.current_stream().cuda_stream
+    g = wl.group
+    for step in range(4):
+        q, k, v = (ref.to_device(a) for a in inp.decode_token(step))
+        out_ref, out_new = torch.empty_like(q), torch.full_like(q, float("nan"))
+        assert b.lola_decode_step(ref.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out_ref.data_ptr(), s) == b.LOLA_OK
+        assert "decode_fused" in ref.last_call_info()["paths"]
+        assert b.lola_decode_step_static(new.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out_new.data_ptr(), s) == b.LOLA_OK
+        assert "decode_fused" not in new.last_call_info()["paths"]
+        torch.cuda.synchronize()
+        a, c = ref.read_state(), new.read_state()
+        assert int(c["status"][0]) == 0
+        resync = False
+        for bi in range(wl.batch):
+            for h in range(wl.n_kv_heads):
+                if set(a["sparse_pos"][bi, h].tolist()) != set(c["sparse_pos"][bi, h].tolist()):
+                    kept, folded = a["threshold"][bi, h]
+                    assert abs(kept - folded) <= 1e-4 * max(1.0, abs(kept)), (step, bi, h, kept, folded)
+                    resync = True
+                    continue
+                err = (out_new[bi, h * g:(h + 1) * g].float() - out_ref[bi, h * g:(h + 1) * g].float()).abs().max().item()
+                assert err <= 2e-2, (step, bi, h, err)
+                assert np.abs(c["H"][bi, h] - a["H"][bi, h]).max() <= 2e-2
+        for key in ("window_k", "window_v", "n_seen"):
+            assert np.array_equal(a[key], c[key]), key
+        if resync:
+            new.write_state(a)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_static_scratch_decode_matches_decode(dtype):
     wl = small_case("noalloc", batch=3, n_q_heads=4, n_kv_heads=2, head_dim=64, feat_half=64, tokens=256, chunk=32,
