@@ -390,7 +390,10 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
         chk["what"] = f"outputs of chunk {ci} left by the timed loop vs the float64 oracle, batch rows {srows}"
         chk["status"] = 0
         res["check"] = chk
-        assert chk["units_within_tol"] >= 0.9 * chk["units"], f"timed outputs disagree with the oracle: {chk}"
+        # (a unit that took the other side of a near-tie earlier in the sample holds a different, equally valid
+        # sparse cache and may miss the tolerance; a wrong kernel misses it everywhere and by far)
+        assert chk["units_within_tol"] >= 0.75 * chk["units"] and chk["worst_abs_err"] < 0.25, \
+            f"timed outputs disagree with the oracle: {chk}"
     layer.close()
     return res
 
@@ -530,7 +533,8 @@ def bench_decode(wl, args, rank, local_rank, world, peaks):
                        f"{T}-token state, batch row {rows[0]} (per unit: worst over the steps)")
         chk["status"] = 0
         res["check"] = chk
-        assert chk["units_within_tol"] >= 0.75 * chk["units"], f"timed outputs disagree with the oracle: {chk}"
+        assert chk["units_within_tol"] >= 0.75 * chk["units"] and chk["worst_abs_err"] < 0.25, \
+            f"timed outputs disagree with the oracle: {chk}"
     layer.close()
     return res
 
