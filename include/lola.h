@@ -60,10 +60,6 @@ typedef enum { LOLA_PHI_SOFTMAX = 0, LOLA_PHI_EXP = 1 } lola_phi;
 /* config flag: run the shape-generic CUDA-core kernels even where tensor-core kernels exist (bf16,
  * F = 64).  Both compute the same function; the flag exists for cross-checks and timing.        */
 #define LOLA_FLAG_GENERIC_KERNELS 1u
-/* config flag: run the fused generation step with one thread block per unit instead of persistent blocks
- * that work through several units (same arithmetic; for cross-checks and timing).                  */
-#define LOLA_FLAG_DECODE_BLOCK_PER_UNIT 2u
-#define LOLA_FLAGS_ALL (LOLA_FLAG_GENERIC_KERNELS | LOLA_FLAG_DECODE_BLOCK_PER_UNIT)
 
 typedef struct lola_config {
   int32_t batch;         /* B >= 1                                                              */
@@ -80,7 +76,7 @@ typedef struct lola_config {
                             contraction and folds the rounded phi(K) (Eq. 13).                  */
   int32_t phi_kind;      /* lola_phi                                                            */
   float softmax_scale;   /* 0 => 1/sqrt(head_dim) (Eq. 2)                                       */
-  uint32_t flags;        /* 0, or an OR of LOLA_FLAG_*                                          */
+  uint32_t flags;        /* 0, or LOLA_FLAG_GENERIC_KERNELS                                     */
 } lola_config;
 
 /* Opaque host-side handle.  Owns no device memory. */
@@ -253,8 +249,7 @@ enum {
   LOLA_PATH_UPDATE_GENERIC = 1u << 8,
   LOLA_PATH_DECODE_FUSED = 1u << 9,      /* the generation step as one kernel (units of up to 8 row tiles)  */
   LOLA_PATH_DECODE_FUSED_LONG = 1u << 10,/* the same for units of 9 to 16 row tiles                         */
-  LOLA_PATH_H_IMAGE_REBUILD = 1u << 11,  /* the tensor-core operand image of H had to be rebuilt first      */
-  LOLA_PATH_DECODE_PERSISTENT = 1u << 12 /* ... by persistent blocks (one per SM, several units each)        */
+  LOLA_PATH_H_IMAGE_REBUILD = 1u << 11   /* the tensor-core operand image of H had to be rebuilt first      */
 };
 typedef struct lola_call_info {
   uint32_t paths;                        /* OR of LOLA_PATH_*                                               */

@@ -43,9 +43,9 @@ class lola_call_info(C.Structure):
 
 
 PATH_BITS = ["attend_tma", "attend_mma", "attend_generic", "score_tma", "score_mma", "score_generic", "select_kernel",
-             "apply_tma", "update_generic", "decode_fused", "decode_fused_long", "h_image_rebuild", "decode_persistent"]
+             "apply_tma", "update_generic", "decode_fused", "decode_fused_long", "h_image_rebuild"]
 LOLA_STATUS_SELFTEST = 128
-LOLA_FLAG_GENERIC_KERNELS, LOLA_FLAG_DECODE_BLOCK_PER_UNIT = 1, 2
+LOLA_FLAG_GENERIC_KERNELS = 1
 
 
 class LolaError(RuntimeError):

@@ -18,7 +18,6 @@
 #include "lola_attend_tc.cuh"
 #include "lola_decode_tc.cuh"
 #include "lola_decode2_tc.cuh"
-#include "lola_decode3_tc.cuh"
 #include "lola_score2_tc.cuh"
 #include "lola_update2_tc.cuh"
 #include "lola_attend2_tc.cuh"
@@ -44,7 +43,7 @@ bool config_ok(const lola_config* c) {
   if ((int64_t)c->sparse + c->max_chunk > 16384) return false;
   if (c->dtype != LOLA_F32 && c->dtype != LOLA_BF16) return false;
   if (c->phi_kind != LOLA_PHI_SOFTMAX && c->phi_kind != LOLA_PHI_EXP) return false;
-  if (!(c->softmax_scale >= 0.f) || (c->flags & ~(uint32_t)LOLA_FLAGS_ALL) != 0) return false;
+  if (!(c->softmax_scale >= 0.f) || (c->flags & ~(uint32_t)LOLA_FLAG_GENERIC_KERNELS) != 0) return false;
   if ((int64_t)2 * c->feat_half * c->head_dim > (int64_t)kUpdThreads * kUpdEPT) return false;
   return true;
 }
@@ -379,14 +378,7 @@ int launch_decode_fused(lola_state* st, const Call& c, cudaStream_t s) {
   const int n_tiles = (L.lam / 64 + (L.eta + 63) / 64 + 1) / 2;
   LaunchScope scope(st, LOLA_KERNEL_DECODE, s, n_tiles <= kDec2MaxTiles ? LOLA_PATH_DECODE_FUSED : LOLA_PATH_DECODE_FUSED_LONG, L.B * L.Hkv);
   const uint4* wt = (const uint4*)(st->base + st->lay.wt);
-  if (n_tiles <= kDec2MaxTiles && L.g <= kDec3Q && !(st->cfg.flags & LOLA_FLAG_DECODE_BLOCK_PER_UNIT)) {
-    // persistent blocks: one per SM, each works through its units with the next unit's set-up under way
-    const int grid = std::min(L.B * L.Hkv, st->sm_count);
-    st->info.paths |= LOLA_PATH_DECODE_PERSISTENT;
-    k_decode3_tc<DPL><<<grid, kDec2Threads, DecodeSmem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, wt);
-    return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
-  }
-  if (n_tiles <= kDec2MaxTiles) {          // one block per unit; longer units run the two-row-group kernel
+  if (n_tiles <= kDec2MaxTiles) {          // the pipelined kernel; longer units run the two-row-group kernel
     if (L.g <= 4)
       k_decode2_tc<DPL, 4><<<L.B * L.Hkv, kDec2Threads, DecodeSmem<DPL>::bytes, s>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, wt);
     else
@@ -518,7 +510,6 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       e[4] = cudaFuncSetAttribute(k_attend2_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<4>::bytes);
       e[5] = cudaFuncSetAttribute(k_decode2_tc<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
       e[6] = cudaFuncSetAttribute(k_decode2_tc<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
-      e[7] = cudaFuncSetAttribute(k_decode3_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<4>::bytes);
     } else {
       e[0] = cudaFuncSetAttribute(k_decode_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[1] = cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
@@ -527,9 +518,8 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       e[4] = cudaFuncSetAttribute(k_attend2_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Attend2Smem<2>::bytes);
       e[5] = cudaFuncSetAttribute(k_decode2_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
       e[6] = cudaFuncSetAttribute(k_decode2_tc<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
-      e[7] = cudaFuncSetAttribute(k_decode3_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DecodeSmem<2>::bytes);
     }
-    for (int i = 0; i < 8; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
+    for (int i = 0; i < 7; ++i) if (e[i] != cudaSuccess) st->have_maps = false;   // the older kernel chain serves every shape
     // one shared-memory carve-out for the kernels that follow each other in a step: a change of the
     // carve-out between two launches costs idle time on every SM
     const int co = (int)cudaSharedmemCarveoutMaxShared;
@@ -538,7 +528,6 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       cudaFuncSetAttribute(k_decode_tc<4, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_decode2_tc<4, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_decode2_tc<4, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
-      cudaFuncSetAttribute(k_decode3_tc<4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_score2_tc<4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_update2_tc<4, 2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_attend2_tc<4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
@@ -547,7 +536,6 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
       cudaFuncSetAttribute(k_decode_tc<2, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_decode2_tc<2, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_decode2_tc<2, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
-      cudaFuncSetAttribute(k_decode3_tc<2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_score2_tc<2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_update2_tc<2, 2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);
       cudaFuncSetAttribute(k_attend2_tc<2>, cudaFuncAttributePreferredSharedMemoryCarveout, co);

@@ -96,9 +96,9 @@ def test_fused_decode_group_sizes(g, batch, mode):
     ("one_tile", 40, 8, 4, 128, 32, 64),       # a unit is a single row tile: set-up, tile and end of neighbouring units overlap
     ("d64", 38, 8, 1, 64, 64, 192),
 ])
-def test_persistent_decode_many_units(name, batch, hkv, g, d, eta, lam):
-    """More units than SMs: the persistent generation kernel works through several units per block, with the
-    set-up of the next unit under way while the current one is scored."""
+def test_fused_decode_many_units(name, batch, hkv, g, d, eta, lam):
+    """More units than SMs in one launch of the fused generation step (several waves of blocks), with units of
+    one and two row tiles."""
     tokens = ((lam + eta) // 64 + 2) * 64
     wl = small_case(f"persist_{name}", batch=batch, n_q_heads=hkv * g, n_kv_heads=hkv, head_dim=d, feat_half=64,
                     tokens=tokens, chunk=64, window=eta, sparse=lam, dtype="bf16", seed=37, decode_steps=6)
@@ -107,12 +107,12 @@ def test_persistent_decode_many_units(name, batch, hkv, g, d, eta, lam):
         ls.prefill(t0, 64, want_out=False, check_state=("members" if t0 + 64 < tokens else True))
     for sidx in range(wl.decode_steps):
         ls.decode(sidx)
-        assert "decode_persistent" in ls.layer.last_call_info()["paths"]
+        assert "decode_fused" in ls.layer.last_call_info()["paths"]
     summ = ls.summary()
     assert summ["resyncs"] <= resync_cap(summ), summ
 
 
-def test_persistent_decode_at_cfg3_shapes_two_units_per_block():
+def test_fused_decode_at_cfg3_shapes_more_units_than_sms():
     """160 units of the decode workload's shapes (7 row tiles per unit) on 148 SMs after a shortened prefill."""
     wl = WORKLOADS["cfg3"].with_(batch=20, tokens=2048, decode_steps=8)
     ls = Lockstep(wl, threads=16, oracle_mode="mirror")
@@ -122,17 +122,6 @@ def test_persistent_decode_at_cfg3_shapes_two_units_per_block():
         ls.decode(sidx)
     summ = ls.summary()
     assert summ["resyncs"] <= resync_cap(summ), summ
-
-
-def test_block_per_unit_decode_flag():
-    """The same step with one thread block per unit (config flag) meets the same bar."""
-    from paper_2505_23666_b200 import binding as b
-    wl = small_case("per_unit", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=384, chunk=64,
-                    window=64, sparse=128, dtype="bf16", seed=13, decode_steps=10)
-    ls = Lockstep(wl, threads=1, oracle_mode="mirror", flags=b.LOLA_FLAG_DECODE_BLOCK_PER_UNIT)
-    summ = drive(ls, 384, 64, 10)
-    assert "decode_persistent" not in ls.layer.last_call_info()["paths"]
-    assert summ["resyncs"] <= 2, summ
 
 
 @pytest.mark.parametrize("mode", BF16_MODES)
