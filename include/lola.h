@@ -15,10 +15,9 @@
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are ordinary
  *     host memory.  The library never allocates or frees device memory; the caller owns every
  *     buffer (state, W, q, k, v, out) and must keep W and the state buffer alive for the life of
- *     the handle.  A handle of a bf16 layer holds two host-side objects of its own, a second
- *     non-blocking stream and a pair of events: lola_prefill_chunk uses them to run the scoring of
- *     the eligible set beside the attention kernel (both only read the memories) and joins them
- *     on the caller's stream before anything is written, so the caller sees one ordered stream.
+ *     the handle.  Everything a call enqueues goes to the caller's stream; inside a lola_prefill_chunk call
+ *     the scoring of the eligible set runs beside the attention kernel (both only read the memories; the
+ *     kernels are chained by programmatic dependent launches on that one stream), and the fold follows both.
  *   - Work is enqueued on the given stream (a cudaStream_t passed as void*; NULL = legacy default
  *     stream) and the call returns without synchronising unless stated otherwise.  All calls on
  *     one state must be issued on one stream, or be ordered by the caller.
@@ -60,6 +59,15 @@ typedef enum { LOLA_PHI_SOFTMAX = 0, LOLA_PHI_EXP = 1 } lola_phi;
 /* config flag: run the shape-generic CUDA-core kernels even where tensor-core kernels exist (bf16,
  * F = 64).  Both compute the same function; the flag exists for cross-checks and timing.        */
 #define LOLA_FLAG_GENERIC_KERNELS 1u
+/* config flags of the cache ablation (appendix "Sparse Cache & Linear Attention Ablation"): the memories are
+ * updated as always, but the queries do not see the linear-attention state (the phi(q)^T H and phi(q)^T s terms
+ * of Eq. 14 are left out) and / or the sparse cache (its sum in Eq. 14 is left out).  With both set Eq. 14 is
+ * softmax attention over the sliding window (and, in a prefill call, the chunk itself).  A query that then sees
+ * nothing at all (window = 0 in a generation step) has no defined output.  Generation steps with either flag run
+ * as the kernel chain, not as the fused kernel.                                                          */
+#define LOLA_FLAG_QUERY_NO_LINEAR 4u
+#define LOLA_FLAG_QUERY_NO_SPARSE 8u
+#define LOLA_FLAGS_ALL (LOLA_FLAG_GENERIC_KERNELS | LOLA_FLAG_QUERY_NO_LINEAR | LOLA_FLAG_QUERY_NO_SPARSE)
 
 typedef struct lola_config {
   int32_t batch;         /* B >= 1                                                              */
@@ -76,7 +84,7 @@ typedef struct lola_config {
                             contraction and folds the rounded phi(K) (Eq. 13).                  */
   int32_t phi_kind;      /* lola_phi                                                            */
   float softmax_scale;   /* 0 => 1/sqrt(head_dim) (Eq. 2)                                       */
-  uint32_t flags;        /* 0, or LOLA_FLAG_GENERIC_KERNELS                                     */
+  uint32_t flags;        /* 0, or an OR of LOLA_FLAG_*                                          */
 } lola_config;
 
 /* Opaque host-side handle.  Owns no device memory. */
@@ -136,6 +144,16 @@ int lola_reset_state(lola_state* st, void* stream);
  * Errors: ARG, SHAPE, ALIGN, CUDA.                                                              */
 int lola_prefill_chunk(lola_state* st, const void* q, const void* k, const void* v, int32_t n_tokens,
                        void* out, void* stream);
+
+/* A run of `n_chunks` consecutive prefill chunks of `n_tokens` tokens each in one call (section "Chunkwise
+ * Inference": the chunks of a prompt in order; the chunk recurrence is sequential, so the run is enqueued chunk
+ * after chunk on `stream`, the kernels of neighbouring chunks overlapping where their dependencies allow).
+ * q, k, v, out hold the chunks one after the other: chunk c is the tensor [B, n_tokens, heads, d] that
+ * lola_prefill_chunk takes, at byte offset c * (bytes of that tensor), all in device memory.  out (and then q)
+ * may be NULL.  Same results, bit for bit, as n_chunks calls of lola_prefill_chunk.
+ * Errors: as lola_prefill_chunk, plus SHAPE for n_chunks < 1; the run stops at the first failing chunk.    */
+int lola_prefill_chunks(lola_state* st, const void* q, const void* k, const void* v, int32_t n_chunks, int32_t n_tokens,
+                        void* out, void* stream);
 
 /* Generation step (Eq. 11-14): update, then attend.  The new pair enters the window; if the window
  * overflows its oldest pair is evicted, E = G u {evicted} is scored against the current H, s, the

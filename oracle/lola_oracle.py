@@ -31,6 +31,10 @@ Readings taken where the paper is silent:
     stays float64 and Eq. 13 folds phi(k) itself.  Tests use it beside the default
     to tell operand rounding apart from arithmetic mistakes.
 
+Cache ablation (appendix "Sparse Cache & Linear Attention Ablation"): `query_linear=False` leaves the
+phi(q)^T H and phi(q)^T s terms out of Eq. 14, `query_sparse=False` the sum over the sparse cache; the
+memories are updated as always.
+
 Parity pins: every function here is pinned by tests/test_oracle_pins.py
 (closed forms, brute force, library special cases).  The absolute values of
 outputs on the five full workloads have no external reference: for those,
@@ -64,6 +68,10 @@ class OracleConfig:
     softmax_scale: Optional[float] = None   # None => 1/sqrt(head_dim) (Eq. 2)
     operand_rounding: str = "none"   # "none" | "bf16"
     schedule: str = "eager"          # "eager" | "lazy" (pseudo-code order of update_chunk)
+    # cache ablation (appendix "Sparse Cache & Linear Attention Ablation"): what the QUERIES see in Eq. 14;
+    # the memories are updated the same way whatever these say
+    query_linear: bool = True        # the phi(q)^T H and phi(q)^T s terms
+    query_sparse: bool = True        # the sum over the sparse cache G
 
     @property
     def group(self) -> int:
@@ -197,7 +205,7 @@ class UnitState:
         z = np.where(visible, z, -np.inf)
         m = np.maximum(0.0, z.max(axis=1, initial=-np.inf))
         w = np.exp(z - m[:, None])                          # masked entries: exp(-inf) = 0
-        lin = np.exp(-m)
+        lin = np.exp(-m) if self.cfg.query_linear else np.zeros_like(m)
         num = lin[:, None] * (fq @ self.H) + w @ V
         den = lin * (fq @ self.s) + w.sum(axis=1)
         return num / den[:, None]
@@ -226,9 +234,10 @@ class UnitState:
         if cfg.schedule == "lazy":                          # pseudo-code order: evict first, then append
             over = max(0, len(self.win_pos) - cfg.window)
             self.evict(*self._pop_oldest(over))
-        K = np.concatenate([self.G_k, self.win_k, k], axis=0)
-        V = np.concatenate([self.G_v, self.win_v, v], axis=0)
-        n_old = len(self.G_pos) + len(self.win_pos)
+        Gk, Gv = (self.G_k, self.G_v) if cfg.query_sparse else (self.G_k[:0], self.G_v[:0])
+        K = np.concatenate([Gk, self.win_k, k], axis=0)
+        V = np.concatenate([Gv, self.win_v, v], axis=0)
+        n_old = len(Gk) + len(self.win_pos)
         vis = np.ones((n, n_old + n), dtype=bool)
         vis[:, n_old:] = np.tril(np.ones((n, n), dtype=bool))
         out = np.stack([self.attend_rows(q[h], K, V, vis) for h in range(g)], axis=0)
@@ -249,8 +258,9 @@ class UnitState:
         self.n_seen += 1
         over = max(0, len(self.win_pos) - cfg.window)
         self.evict(*self._pop_oldest(over))
-        K = np.concatenate([self.G_k, self.win_k], axis=0)
-        V = np.concatenate([self.G_v, self.win_v], axis=0)
+        Gk, Gv = (self.G_k, self.G_v) if cfg.query_sparse else (self.G_k[:0], self.G_v[:0])
+        K = np.concatenate([Gk, self.win_k], axis=0)
+        V = np.concatenate([Gv, self.win_v], axis=0)
         vis = np.ones((q.shape[0], K.shape[0]), dtype=bool)
         return self.attend_rows(q, K, V, vis)
 

@@ -45,7 +45,7 @@ class lola_call_info(C.Structure):
 PATH_BITS = ["attend_tma", "attend_mma", "attend_generic", "score_tma", "score_mma", "score_generic", "select_kernel",
              "apply_tma", "update_generic", "decode_fused", "decode_fused_long", "h_image_rebuild"]
 LOLA_STATUS_SELFTEST = 128
-LOLA_FLAG_GENERIC_KERNELS = 1
+LOLA_FLAG_GENERIC_KERNELS, LOLA_FLAG_QUERY_NO_LINEAR, LOLA_FLAG_QUERY_NO_SPARSE = 1, 4, 8
 
 
 class LolaError(RuntimeError):
@@ -65,6 +65,7 @@ def _load() -> C.CDLL:
         "lola_state_bytes": (sz, [cfgp]),
         "lola_init_state": (C.c_int, [cfgp, vp, vp, sz, vp, C.POINTER(vp)]),
         "lola_prefill_chunk": (C.c_int, [vp, vp, vp, vp, i32, vp, vp]),
+        "lola_prefill_chunks": (C.c_int, [vp, vp, vp, vp, i32, i32, vp, vp]),
         "lola_decode_step": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "lola_decode_step_static": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "lola_staging_bytes": (sz, [cfgp, i32]),
@@ -91,7 +92,7 @@ def _load() -> C.CDLL:
 
 
 _lib = _load()
-EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_decode_step", "lola_decode_step_static", "lola_staging_bytes",
+EXPORTS = ["lola_state_bytes", "lola_init_state", "lola_prefill_chunk", "lola_prefill_chunks", "lola_decode_step", "lola_decode_step_static", "lola_staging_bytes",
            "lola_prefill_chunk_host", "lola_decode_step_host", "lola_prefill_host", "lola_read_state", "lola_write_state",
            "lola_reset_state", "lola_profile_enable", "lola_profile_read", "lola_last_call_info", "lola_selftest_wait_timeout",
            "lola_launch_count", "lola_tokens_seen", "lola_set_tokens_seen", "lola_destroy_state", "lola_strerror"]
@@ -121,6 +122,10 @@ def lola_init_state(cfg: lola_config, W_dev: int, state_dev: int, state_bytes: i
 
 def lola_prefill_chunk(st: int, q: int, k: int, v: int, n_tokens: int, out: int, stream: int) -> int:
     return _lib.lola_prefill_chunk(st, q or None, k, v, int(n_tokens), out or None, stream)
+
+
+def lola_prefill_chunks(st: int, q: int, k: int, v: int, n_chunks: int, n_tokens: int, out: int, stream: int) -> int:
+    return _lib.lola_prefill_chunks(st, q or None, k, v, int(n_chunks), int(n_tokens), out or None, stream)
 
 
 def lola_decode_step(st: int, q: int, k: int, v: int, out: int, stream: int) -> int:
@@ -261,6 +266,15 @@ class LolaLayer:
         _check(lola_prefill_chunk(self.handle, q.data_ptr() if (want_out and q is not None) else 0, k.data_ptr(),
                                   v.data_ptr(), n, out.data_ptr() if want_out else 0, self._stream()),
                "lola_prefill_chunk")
+        return out if want_out else None
+
+    def prefill_chunks(self, q, k, v, out=None, want_out=True):
+        """q, k, v (and out): device tensors [n_chunks, B, n_tokens, heads, d], the chunks in order."""
+        nch, n = k.shape[0], k.shape[2]
+        if want_out and out is None:
+            out = torch.empty_like(q)
+        _check(lola_prefill_chunks(self.handle, q.data_ptr() if want_out else 0, k.data_ptr(), v.data_ptr(), nch, n,
+                                   out.data_ptr() if want_out else 0, self._stream()), "lola_prefill_chunks")
         return out if want_out else None
 
     def decode_step(self, q, k, v, out=None):

@@ -43,7 +43,7 @@ bool config_ok(const lola_config* c) {
   if ((int64_t)c->sparse + c->max_chunk > 16384) return false;
   if (c->dtype != LOLA_F32 && c->dtype != LOLA_BF16) return false;
   if (c->phi_kind != LOLA_PHI_SOFTMAX && c->phi_kind != LOLA_PHI_EXP) return false;
-  if (!(c->softmax_scale >= 0.f) || (c->flags & ~(uint32_t)LOLA_FLAG_GENERIC_KERNELS) != 0) return false;
+  if (!(c->softmax_scale >= 0.f) || (c->flags & ~(uint32_t)LOLA_FLAGS_ALL) != 0) return false;
   if ((int64_t)2 * c->feat_half * c->head_dim > (int64_t)kUpdThreads * kUpdEPT) return false;
   return true;
 }
@@ -173,8 +173,6 @@ struct lola_state {
   int sm_count = 0;                    // SMs of the device (grid of the persistent generation kernel)
   bool have_maps = false;              // TMA descriptors of the sparse cache and the window ring exist
   bool himg_valid = false;             // the bf16 operand image of H matches H
-  cudaStream_t aux = nullptr;          // second stream: Eq. 10 scoring runs beside the attention kernel
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   // lola_prefill_host: two copy streams and the events that order them against the kernels (made at first use)
   cudaStream_t cp_in = nullptr, cp_out = nullptr;
   cudaEvent_t ev_start = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
@@ -236,8 +234,11 @@ int ensure_h_image(lola_state* st, cudaStream_t s) {
   return LOLA_OK;
 }
 
+// before_scoring: the kernel after this one in the stream is the scoring kernel of the same call, which only
+// reads the memories and runs beside this one: it is let go once this kernel has seen everything before it
+// complete, and it waits for this kernel at its end (so that whatever follows sees both complete).
 template <typename T, int DPL>
-int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
+int launch_attend(lola_state* st, const Call& c, cudaStream_t s, bool before_scoring = false) {
   const Layer& L = st->L;
   dim3 grid((L.g * c.nq + kAttRows - 1) / kAttRows, L.B * L.Hkv);
   if (st->have_maps && !st->force_chain && c.att_chunk == c.nq && c.nq <= 64 && c.n == c.nq) {
@@ -250,7 +251,7 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s) {
       LaunchScope scope(st, LOLA_KERNEL_ATTEND, s, LOLA_PATH_ATTEND_TMA, (int)(grid2.x * grid2.y));
       const cudaError_t le = launch_pdl(k_attend2_tc<DPL>, grid2, dim3(kAt2Threads), Attend2Smem<DPL>::bytes, s, L, c, st->tm_gk, st->tm_gv,
                                         st->tm_wk, st->tm_wv, tq, tk, tv, tout, (const uint4*)(st->base + st->lay.wt),
-                                        (const __nv_bfloat16*)(st->base + st->lay.himg));
+                                        (const __nv_bfloat16*)(st->base + st->lay.himg), before_scoring ? 1 : 0);
       return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
     }
   }
@@ -272,7 +273,7 @@ inline bool fast_update_path(const lola_state* st, const Call& c) {
 
 // Eq. 10 scoring and the top-lambda selection on TMA-fed tensor-core kernels.  Both only read the
 // memories (scores, positions) and write scores / work lists, so they may run beside the attention
-// kernel on another stream.
+// kernel (busy_sms > 0: that kernel precedes this one in the stream and this one is its programmatic dependent).
 template <int DPL>
 int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss, int busy_sms = 0) {
   const Layer& L = st->L;
@@ -293,8 +294,9 @@ int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss, int busy
   // the selection (Eq. 12) runs in the scoring kernel: the last block of a unit to finish does it
   dim3 grid((NT + tpc - 1) / tpc, U);
   LaunchScope scope(st, LOLA_KERNEL_SCORE, ss, LOLA_PATH_SCORE_TMA, (int)(grid.x * grid.y));
-  k_score2_tc<DPL><<<grid, kSc2Threads, Score2Smem<DPL>::bytes, ss>>>(L, c, st->tm_gk, st->tm_gv, st->tm_wk, st->tm_wv, img, himg, tpc);
-  return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
+  const cudaError_t le = launch_pdl(k_score2_tc<DPL>, grid, dim3(kSc2Threads), Score2Smem<DPL>::bytes, ss, L, c, st->tm_gk, st->tm_gv, st->tm_wk,
+                                    st->tm_wv, img, (const __nv_bfloat16*)himg, tpc, busy_sms > 0 ? 1 : 0);
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
 // Eq. 13 fold, moves into the sparse cache and window roll from the selection's work lists; keeps the
@@ -350,21 +352,17 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
 template <typename T, int DPL>
 int run_prefill(lola_state* st, Call c, cudaStream_t s) {
   int rc = LOLA_OK;
-  // Attention and scoring both only read the memories: with outputs wanted and the tensor-core update
-  // path in use, the scoring kernel runs on the handle's second stream beside the attention kernel
-  // and the selection joins the two.
-  if (c.out && st->aux && fast_update_path(st, c)) {
+  // Attention and scoring both only read the memories: with outputs wanted and the tensor-core update path
+  // in use they run side by side, all on the caller's stream, chained by programmatic dependent launches:
+  // the attention kernel waits for everything before it and then lets the scoring kernel (with the selection
+  // in its last block per unit) start; the scoring kernel waits for the attention kernel only at its end; the
+  // fold waits for the scoring kernel, hence for both.
+  if (c.out && fast_update_path(st, c)) {
     if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
-    if (cudaEventRecord(st->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(st->aux, st->ev_fork, 0) != cudaSuccess)
-      return LOLA_ERR_CUDA;
-    // scoring and selection are enqueued first: their many short CTAs take the SMs at once and the
-    // attention CTAs fill in as they drain; the fold joins both
-    rc = launch_score_select<DPL>(st, c, st->aux, (((st->L.g + 1) / 2 + 1) / 2) * st->L.B * st->L.Hkv);
+    rc = launch_attend<T, DPL>(st, c, s, true);
     if (rc != LOLA_OK) return rc;
-    rc = launch_attend<T, DPL>(st, c, s);
+    rc = launch_score_select<DPL>(st, c, s, (((st->L.g + 1) / 2 + 1) / 2) * st->L.B * st->L.Hkv);
     if (rc != LOLA_OK) return rc;
-    if (cudaEventRecord(st->ev_join, st->aux) != cudaSuccess || cudaStreamWaitEvent(s, st->ev_join, 0) != cudaSuccess)
-      return LOLA_ERR_CUDA;
     return launch_apply<DPL>(st, c, s);
   }
   if (c.out) rc = launch_attend<T, DPL>(st, c, s);
@@ -397,7 +395,8 @@ int launch_decode_fused(lola_state* st, const Call& c, cudaStream_t s) {
 template <typename T, int DPL>
 int run_decode(lola_state* st, Call c, cudaStream_t s) {
   // steady state (caches full, one pair leaves the window): the whole step is one kernel
-  if (st->fused_decode && !st->force_chain && c.mode == UPD_SELECT && c.r == 1 && c.count_g == st->L.lam)
+  const bool ablation = (st->cfg.flags & (LOLA_FLAG_QUERY_NO_LINEAR | LOLA_FLAG_QUERY_NO_SPARSE)) != 0;
+  if (st->fused_decode && !st->force_chain && !ablation && c.mode == UPD_SELECT && c.r == 1 && c.count_g == st->L.lam)
   {
     st->himg_valid = false;              // the fused step folds into H only
     return launch_decode_fused<DPL>(st, c, s);
@@ -542,16 +541,6 @@ int lola_init_state(const lola_config* cfg, const void* W_dev, void* state_dev, 
     }
     cudaGetLastError();   // a refused preference is not an error
   }
-  if (rc == LOLA_OK && st->have_maps) {
-    // host-side objects only (no device memory): a second stream and two events to run the scoring
-    // kernel beside the attention kernel; without them everything stays on the caller's stream
-    if (cudaStreamCreateWithFlags(&st->aux, cudaStreamNonBlocking) != cudaSuccess) st->aux = nullptr;
-    if (st->aux && (cudaEventCreateWithFlags(&st->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-                    cudaEventCreateWithFlags(&st->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
-      cudaStreamDestroy(st->aux);
-      st->aux = nullptr;
-    }
-  }
   // one-kernel generation step: lambda a whole number of 64-row blocks, the row stream within 16 tiles
   st->fused_decode = st->have_maps && cfg->sparse >= 64 && cfg->sparse % 64 == 0 && L.g <= kDecQ &&
                      (cfg->sparse / 64 + (cfg->window + 63) / 64 + 1) / 2 <= kDecMaxTiles;
@@ -597,10 +586,29 @@ int lola_prefill_chunk(lola_state* st, const void* q, const void* k, const void*
   c.q = q; c.k = k; c.v = v; c.out = out;
   c.n = n_tokens; c.nq = n_tokens; c.n_seen = (int)st->n_seen;
   c.r = g.r; c.r_pos0 = g.r_pos0; c.count_g = g.count_g; c.mode = g.mode;
-  c.att_g = g.count_g; c.att_w0 = (int)st->n_seen - g.cw; c.att_wn = g.cw; c.att_chunk = n_tokens;
+  c.att_g = (st->cfg.flags & LOLA_FLAG_QUERY_NO_SPARSE) ? 0 : g.count_g;
+  c.att_w0 = (int)st->n_seen - g.cw; c.att_wn = g.cw; c.att_chunk = n_tokens;
+  c.att_flags = (st->cfg.flags & LOLA_FLAG_QUERY_NO_LINEAR) ? 1 : 0;
   int rc = LOLA_DISPATCH(run_prefill, st, c, (cudaStream_t)stream);
   if (rc == LOLA_OK) st->n_seen += n_tokens;
   return rc;
+}
+
+int lola_prefill_chunks(lola_state* st, const void* q, const void* k, const void* v, int32_t n_chunks, int32_t n_tokens,
+                        void* out, void* stream) {
+  if (!st || !k || !v) return LOLA_ERR_ARG;
+  if (out && !q) return LOLA_ERR_ARG;
+  if (n_chunks < 1 || n_tokens < 1 || n_tokens > st->cfg.max_chunk) return LOLA_ERR_SHAPE;
+  const lola_config& c = st->cfg;
+  const size_t es = c.dtype == LOLA_BF16 ? 2 : 4;
+  const size_t qbytes = (size_t)c.batch * n_tokens * c.n_q_heads * c.head_dim * es;
+  const size_t kbytes = (size_t)c.batch * n_tokens * c.n_kv_heads * c.head_dim * es;
+  for (int i = 0; i < n_chunks; ++i) {
+    const int rc = lola_prefill_chunk(st, out ? (const char*)q + (size_t)i * qbytes : nullptr, (const char*)k + (size_t)i * kbytes,
+                                      (const char*)v + (size_t)i * kbytes, n_tokens, out ? (char*)out + (size_t)i * qbytes : nullptr, stream);
+    if (rc != LOLA_OK) return rc;
+  }
+  return LOLA_OK;
 }
 
 int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v, void* out, void* stream) {
@@ -614,7 +622,9 @@ int lola_decode_step(lola_state* st, const void* q, const void* k, const void* v
   c.n = 1; c.nq = 1; c.n_seen = (int)st->n_seen;
   c.r = g.r; c.r_pos0 = g.r_pos0; c.count_g = g.count_g; c.mode = g.mode;
   const int cw_after = (int)std::min<int64_t>(st->cfg.window, st->n_seen + 1);
-  c.att_g = g.new_count_g; c.att_w0 = (int)(st->n_seen + 1) - cw_after; c.att_wn = cw_after; c.att_chunk = 0;
+  c.att_g = (st->cfg.flags & LOLA_FLAG_QUERY_NO_SPARSE) ? 0 : g.new_count_g;
+  c.att_w0 = (int)(st->n_seen + 1) - cw_after; c.att_wn = cw_after; c.att_chunk = 0;
+  c.att_flags = (st->cfg.flags & LOLA_FLAG_QUERY_NO_LINEAR) ? 1 : 0;
   int rc = LOLA_DISPATCH(run_decode, st, c, (cudaStream_t)stream);
   if (rc == LOLA_OK) st->n_seen += 1;
   return rc;
@@ -876,9 +886,6 @@ int lola_destroy_state(lola_state* st) {
   if (!st) return LOLA_ERR_ARG;
   for (auto* v : {&st->records, &st->pool})
     for (ProfRecord& r : *v) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
-  if (st->aux) { cudaStreamSynchronize(st->aux); cudaStreamDestroy(st->aux); }
-  if (st->ev_fork) cudaEventDestroy(st->ev_fork);
-  if (st->ev_join) cudaEventDestroy(st->ev_join);
   if (st->cp_in) { cudaStreamSynchronize(st->cp_in); cudaStreamDestroy(st->cp_in); }
   if (st->cp_out) { cudaStreamSynchronize(st->cp_out); cudaStreamDestroy(st->cp_out); }
   for (cudaEvent_t e : {st->ev_start, st->ev_in[0], st->ev_in[1], st->ev_done[0], st->ev_done[1], st->ev_out[0], st->ev_out[1]})

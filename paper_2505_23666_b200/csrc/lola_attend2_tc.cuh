@@ -59,7 +59,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
              const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
              const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_ck,
              const __grid_constant__ CUtensorMap tm_cv, const __grid_constant__ CUtensorMap tm_out, const uint4* wt_image,
-             const __nv_bfloat16* ht_image) {
+             const __nv_bfloat16* ht_image, int before_scoring) {
   using S = Attend2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
@@ -99,11 +99,15 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
-  if (tid == 0) tc::grid_dep_launch_dependents();    // the next kernel may set itself up beside this one
+  // the next kernel may set itself up beside this one.  before_scoring: the next kernel is the scoring kernel of
+  // the same call, which only reads the memories and starts without waiting: it may only start once this block
+  // has seen everything before it complete (below)
+  if (tid == 0 && !before_scoring) tc::grid_dep_launch_dependents();
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
   tc::grid_dep_wait();                               // everything before this kernel in the stream is complete
+  if (tid == 0 && before_scoring) tc::grid_dep_launch_dependents();
   const uint32_t tmem = X.tmem_slot;
 
   // block `blk` of the key stream -> TMA source
@@ -336,7 +340,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       // into columns 64 + 32 hf .. of S_w (A operand of the linear product)
       float e[64];
       tc::tmem_ld64(tm_s, e);
-      const float em = tc::fast_exp2(-m_used);
+      const float em = (c.att_flags & 1) ? 0.f : tc::fast_exp2(-m_used);   // (0: the queries do not see H, s)
       const float sgn = hf ? -kLog2e : kLog2e;
       float scale;
       if (L.phi_kind == 1) {

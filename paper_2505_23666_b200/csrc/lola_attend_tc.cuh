@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(128) k_attend_tc(Layer L, Call c) {
   tc::fence_after_sync();
 
   {
-    const float e = __expf(-m);
+    const float e = (c.att_flags & 1) ? 0.f : __expf(-m);       // (0: the queries do not see H, s)
     const float inv = 1.0f / fmaf(e, lden, l);
     T* op = nullptr;
     if (row < nrows) {

@@ -297,7 +297,7 @@ __global__ void __launch_bounds__(256) k_attend(Layer L, Call c) {
     int row = row0 + warp * 2 + rr;
     if (row < nrows) {
       int hl = row / c.nq, r = row % c.nq;
-      float e = expf(-m[rr]);
+      float e = (c.att_flags & 1) ? 0.f : expf(-m[rr]);      // (0: the queries do not see H, s)
       float den = fmaf(e, lden[rr], l[rr]);
       T* op = (T*)c.out + (((size_t)b * c.nq + r) * L.Hq + h * L.g + hl) * d;
 #pragma unroll

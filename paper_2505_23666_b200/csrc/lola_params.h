@@ -60,6 +60,7 @@ struct Call {           // one prefill chunk or decode step
   int att_w0;           // first window position the queries see
   int att_wn;           // number of window positions the queries see (all in the ring)
   int att_chunk;        // incoming tokens seen causally straight from k, v (prefill) or 0 (decode)
+  int att_flags;        // bit 0: the queries do not see H, s (the linear terms of Eq. 14 are left out)
 };
 
 }  // namespace lola

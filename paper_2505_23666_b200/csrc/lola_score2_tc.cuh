@@ -47,7 +47,7 @@ template <int DPL>
 __global__ void __launch_bounds__(kSc2Threads, 1)
 k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image,
-            const __nv_bfloat16* ht_image, int tiles_per_cta) {
+            const __nv_bfloat16* ht_image, int tiles_per_cta, int beside_attention) {
   using S = Score2Smem<DPL>;
   if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
@@ -88,6 +88,12 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
   __syncthreads();
+  // Launched as a programmatic dependent, this kernel may be resident while the kernel before it still runs.
+  // beside_attention: that kernel is the attention kernel of the same call, which only reads the memories and has
+  // let this one start after seeing everything before it complete: nothing to wait for here; every block waits
+  // for it at its end instead, so that whatever follows this kernel follows both.
+  if (!beside_attention) tc::grid_dep_wait();
+  if (tid == 0) tc::grid_dep_launch_dependents();
   if (lead && tile0 + wg < tile1) {
     decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile0 + wg, nGB, nRB, unit, bar_k);
     decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile0 + wg, nGB, nRB, unit, bar_v);
@@ -229,6 +235,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   __shared__ int is_last;
   if (gridDim.x == 1) {                              // one block per unit: it has all the unit's scores
     update2_body<DPL, 1>(L, c, wt_image, nullptr, sm, unit);
+    if (beside_attention) tc::grid_dep_wait();
     return;
   }
   if (tid == 0) {
@@ -242,6 +249,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     __threadfence();
     update2_body<DPL, 1>(L, c, wt_image, nullptr, sm, unit);
   }
+  if (beside_attention) tc::grid_dep_wait();
 }
 
 }  // namespace lola

@@ -138,7 +138,8 @@ class Lockstep:
         self.oracle_mode = oracle_mode
         self.tol = tolerances(wl.dtype, oracle_mode)
         self.oracle = oracle_for(wl, self.inputs, B, oracle_mode, threads, softmax_scale=(softmax_scale or None),
-                                 phi_kind=phi_kind)
+                                 phi_kind=phi_kind, query_linear=not (flags & binding.LOLA_FLAG_QUERY_NO_LINEAR),
+                                 query_sparse=not (flags & binding.LOLA_FLAG_QUERY_NO_SPARSE))
         self.ocfg = self.oracle.cfg
         self.cfg = binding.make_config(B, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.feat_half, wl.window,
                                        wl.sparse, max(wl.chunk, 1), dtype=wl.dtype, generic_kernels=generic_kernels,

@@ -194,6 +194,21 @@ def test_bf16_generic_kernels_flag():
     drive(ls, 200, 16, 6)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("no_linear,no_sparse", [(True, False), (False, True), (True, True)])
+def test_query_restriction_flags(no_linear, no_sparse, dtype):
+    """The cache ablation: the queries do not see H, s and / or the sparse cache; the memories are updated as
+    always.  Prefill chunks (tensor-core kernels in bf16, CUDA-core kernels in fp32) and generation steps."""
+    from paper_2505_23666_b200 import binding as b
+    flags = (b.LOLA_FLAG_QUERY_NO_LINEAR if no_linear else 0) | (b.LOLA_FLAG_QUERY_NO_SPARSE if no_sparse else 0)
+    wl = small_case("ablation", batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, feat_half=64, tokens=448, chunk=64,
+                    window=64, sparse=128, dtype=dtype, seed=41, decode_steps=6, scale_a=(0.125 if dtype == "f32" else 1.0))
+    ls = Lockstep(wl, threads=1, oracle_mode="mirror", flags=flags)
+    summ = drive(ls, 448, 64, 6)
+    assert "decode_fused" not in ls.layer.last_call_info()["paths"]
+    assert summ["resyncs"] <= 2, summ
+
+
 def test_exp_feature_map():
     """Eq. 6 as printed, [exp(xW), exp(-xW)], fp32 mode (CUDA-core kernels)."""
     wl = small_case("exp", batch=1, n_q_heads=2, n_kv_heads=2, tokens=160, chunk=16, window=16, sparse=24,
@@ -258,6 +273,12 @@ def test_prefill_host_run_of_chunks():
     for c in range(nch):
         out = b.layer.prefill_chunk(dq[c], dk[c], dv[c])
         assert torch.equal(out.cpu(), hout[c]), f"chunk {c}"
+    # the run of chunks from device memory in one call
+    d2 = Lockstep(wl, threads=1)
+    assert torch.equal(d2.layer.prefill_chunks(dq, dk, dv).cpu(), hout)
+    sd = d2.layer.read_state()
+    for key in ("H", "s", "sparse_pos", "sparse_k", "sparse_v", "window_k", "window_v"):
+        assert np.array_equal(sd[key], b.layer.read_state()[key]), key
     sa, sb = a.layer.read_state(), b.layer.read_state()
     for key in ("H", "s", "sparse_pos", "sparse_k", "sparse_v", "window_k", "window_v"):
         assert np.array_equal(sa[key], sb[key]), key

@@ -467,3 +467,57 @@ def test_zero_feature_weights_running_mean():
         w0 = max(0, t0 - eta)
         wts = np.array([2.0 / F] * w0 + [1.0] * (t + 1 - w0))
         np.testing.assert_allclose(out[0, t], (wts[:, None] * v[:t + 1]).sum(0) / wts.sum(), rtol=1e-12)
+
+
+# ------------------------------------------------------------------ cache ablation (what the queries see)
+@pytest.mark.parametrize("lin,sp", [(True, True), (False, True), (True, False), (False, False)])
+def test_query_restrictions_change_eq14_only(lin, sp):
+    """The ablation's flags leave the memories alone and drop exactly their terms from Eq. 14: outputs are
+    recomputed from the raw arrays, the members' positions and H, s with unshifted exponentials; with both
+    terms hidden the output is textbook softmax attention over the window and the causal part of the chunk."""
+    d, F, eta, lam, C, n = 8, 4, 6, 5, 4, 48
+    rng = np.random.default_rng(77)
+    W = rng.standard_normal((d, F)) / np.sqrt(d)
+    q, k, v = rand_qkv(n, d, 2, rng=rng)
+    q, k, v = 0.5 * q, 0.5 * k, v
+    full = UnitState(OracleConfig(1, 2, 1, d, F, eta, lam), W)
+    abl = UnitState(OracleConfig(1, 2, 1, d, F, eta, lam, query_linear=lin, query_sparse=sp), W)
+    scale = 1.0 / np.sqrt(d)
+    for t0 in range(0, n, C):
+        G_pos, H, s_ = abl.G_pos.copy(), abl.H.copy(), abl.s.copy()
+        w0 = max(0, t0 - eta)
+        out = abl.prefill_chunk(q[:, t0:t0 + C], k[t0:t0 + C], v[t0:t0 + C])
+        full.prefill_chunk(q[:, t0:t0 + C], k[t0:t0 + C], v[t0:t0 + C])
+        # the memories do not depend on what the queries see
+        assert np.array_equal(abl.G_pos, full.G_pos) and np.array_equal(abl.H, full.H) and np.array_equal(abl.s, full.s)
+        for hh in range(2):
+            for r in range(C):
+                t = t0 + r
+                keys = list(range(w0, t + 1)) + (list(map(int, G_pos)) if sp else [])
+                wts = np.exp(scale * (k[keys] @ q[hh, t]))
+                num, den = wts @ v[keys], wts.sum()
+                if lin:
+                    fq = lib_phi(q[hh, t][None], W)[0]
+                    num, den = num + fq @ H, den + fq @ s_
+                np.testing.assert_allclose(out[hh, r], num / den, rtol=1e-10, atol=1e-12)
+                if not lin and not sp:
+                    keys = list(range(w0, t + 1))
+                    ref = scipy.special.softmax(scale * (k[keys] @ q[hh, t])) @ v[keys]
+                    np.testing.assert_allclose(out[hh, r], ref, rtol=1e-10, atol=1e-12)
+    # generation steps: the new pair is in the window, the sparse cache is the updated one
+    for t in range(n - 6, n):
+        pass
+    qd, kd, vd = rand_qkv(6, d, 2, rng=rng)
+    for i in range(6):
+        out = abl.decode_step(0.5 * qd[:, i], 0.5 * kd[i], vd[i])
+        full.decode_step(0.5 * qd[:, i], 0.5 * kd[i], vd[i])
+        assert np.array_equal(abl.G_pos, full.G_pos) and np.array_equal(abl.H, full.H)
+        Ks = np.concatenate([abl.win_k] + ([abl.G_k] if sp else []), axis=0)
+        Vs = np.concatenate([abl.win_v] + ([abl.G_v] if sp else []), axis=0)
+        for hh in range(2):
+            wts = np.exp(scale * (Ks @ (0.5 * qd[hh, i])))
+            num, den = wts @ Vs, wts.sum()
+            if lin:
+                fq = lib_phi(0.5 * qd[hh, i][None], W)[0]
+                num, den = num + fq @ abl.H, den + fq @ abl.s
+            np.testing.assert_allclose(out[hh], num / den, rtol=1e-10, atol=1e-12)
