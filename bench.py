@@ -125,7 +125,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -145,7 +145,10 @@ class ClockSampler:
                 self.proc.kill()
 
     def summary(self, t0, t1):
-        rows = [s for (t, s) in self.samples if t0 <= t <= t1] or [s for (_, s) in self.samples]
+        rows = [s for (t, s) in self.samples if t0 <= t <= t1]
+        if not rows and self.samples:                 # a timed region shorter than the sampling period: the nearest samples
+            mid = 0.5 * (t0 + t1)
+            rows = [s for (_, s) in sorted(self.samples, key=lambda ts: abs(ts[0] - mid))[:3]]
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for row in rows:
@@ -257,6 +260,7 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
     from paper_2505_23666_b200 import binding
     from paper_2505_23666_b200.workloads import WorkloadInputs
     dev = torch.device(f"cuda:{local_rank}")
+    sampler = ClockSampler(local_rank)                            # (started early: the tool takes a while to deliver)
     inputs = WorkloadInputs(wl.with_(batch=wl.batch * world))
     rows = rank_rows(rank, wl.batch)
     B, T, C = wl.batch, wl.tokens, wl.chunk
@@ -290,7 +294,6 @@ def bench_prefill(wl, args, rank, local_rank, world, peaks):
         layer.reset()
         layer.prefill_host(hq, hk, hv, hout)          # all chunks of the prompt; copies overlap the kernels
 
-    sampler = ClockSampler(local_rank)
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize(dev)
@@ -607,7 +610,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
         dist.barrier()
     peaks = load_peaks()
-    default_steps = {"cfg0": 20, "cfg1": 20, "cfg2": 10, "cfg3": 5, "cfg4": 3}
+    default_steps = {"cfg0": 20, "cfg1": 20, "cfg2": 40, "cfg3": 5, "cfg4": 3}
     user_steps = args.steps
     args.steps = user_steps or default_steps[main_name]
     res = (bench_decode if wl.decode_steps else bench_prefill)(wl, args, rank, local_rank, world, peaks)

@@ -77,7 +77,6 @@ __global__ void __launch_bounds__(kDec2Threads, 1)
 k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
              const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image) {
   using S = DecodeSmem<DPL>;
-  if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
   constexpr int F = 64, D = 128;
@@ -120,6 +119,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   auto stage_pt = [&](int i) { return S::stage0 + (uint32_t)i * S::stage_bytes + S::st_pt; };   // offset from sm
 
   // everything the prologue needs from global memory is requested first, so that the round trips overlap
+  const int pre_status = *reinterpret_cast<volatile const int*>(L.status);   // (acted on below: an earlier kernel failed: do nothing)
   float pre_s = 0.f, pre_k = 0.f, pre_v = 0.f;
   uint4 pre_q = make_uint4(0, 0, 0, 0);
   if (tid < D) pre_s = L.s[(size_t)unit * D + tid];
@@ -147,6 +147,10 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
   __syncthreads();
+  if (pre_status != 0) {                             // the state's status word is set: leave the memories as they are
+    if (warp == 0) tc::tmem_dealloc(X.tmem_slot, 512);
+    return;
+  }
   if (tid == 17 * 32) {
     // W^T straight into the operand rows; H (fp32) into the key and value buffers of stage 1, which
     // the second tile only needs later; the first tile starts to stream at once

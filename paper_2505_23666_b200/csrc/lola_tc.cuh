@@ -394,18 +394,50 @@ __device__ __forceinline__ void phi_half(const uint32_t (&u)[64], bool neg, bool
 // takes both parts (two K blocks of one product) where Eq. 10's takes hi alone.
 __device__ __forceinline__ void phi_half_split(const uint32_t (&u)[64], bool neg, bool exp_kind, uint32_t (&hi)[32], uint32_t (&lo)[32]) {
   const float kL = neg ? -1.4426950408889634f : 1.4426950408889634f;
-  float x[64];
-  float mm = -3.0e38f;
+  const uint64_t sc2 = pack_f2(kL, kL);
+  uint64_t x2[32];
 #pragma unroll
-  for (int i = 0; i < 64; ++i) { x[i] = __uint_as_float(u[i]) * kL; mm = fmaxf(mm, x[i]); }
-  if (exp_kind) mm = 0.f;
-  float sum = 0.f;
+  for (int q = 0; q < 32; ++q) x2[q] = mul2(pack_u2(u[2 * q], u[2 * q + 1]), sc2);   // u * kL, in log2 units
+  float mm = 0.f;
+  if (!exp_kind) {
+    float a, b;
+    unpack_f2(x2[0], a, b);
 #pragma unroll
-  for (int i = 0; i < 64; ++i) { x[i] = fast_exp2(x[i] - mm); sum += x[i]; }
-  const float inv = exp_kind ? 1.0f : 1.0f / sum;
+    for (int q = 1; q < 31; q += 2) {
+      float c0, c1, c2, c3;
+      unpack_f2(x2[q], c0, c1);
+      unpack_f2(x2[q + 1], c2, c3);
+      a = max3(a, c0, c1);
+      b = max3(b, c2, c3);
+    }
+    float c0, c1;
+    unpack_f2(x2[31], c0, c1);
+    mm = fmaxf(max3(a, c0, c1), b);
+  }
+  const uint64_t off2 = pack_f2(-mm, -mm);
+  uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = acc0;
+#pragma unroll
+  for (int q = 0; q < 32; q += 2) {
+    float x0, x1, x2f, x3;
+    unpack_f2(add2(x2[q], off2), x0, x1);
+    unpack_f2(add2(x2[q + 1], off2), x2f, x3);
+    x2[q] = pack_f2(fast_exp2(x0), fast_exp2(x1));
+    x2[q + 1] = pack_f2(fast_exp2(x2f), fast_exp2(x3));
+    acc0 = add2(acc0, x2[q]);
+    acc1 = add2(acc1, x2[q + 1]);
+  }
+  float inv = 1.0f;
+  if (!exp_kind) {
+    float s0, s1, s2, s3;
+    unpack_f2(acc0, s0, s1);
+    unpack_f2(acc1, s2, s3);
+    inv = 1.0f / ((s0 + s1) + (s2 + s3));
+  }
+  const uint64_t inv2 = pack_f2(inv, inv);
 #pragma unroll
   for (int q = 0; q < 32; ++q) {
-    const float a = x[2 * q] * inv, b = x[2 * q + 1] * inv;
+    float a, b;
+    unpack_f2(exp_kind ? x2[q] : mul2(x2[q], inv2), a, b);
     __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
     const float2 hf = __bfloat1622float2(h2);
     __nv_bfloat162 l2 = __floats2bfloat162_rn(a - hf.x, b - hf.y);
