@@ -5,8 +5,8 @@
 //   feature group (warps 0-7)   per tile: q.k columns and their warp maxima into shared memory, the
 //                               feature map of U into tensor memory; no barrier inside the group
 //   score group   (warps 8-15)  per tile: running maxima and softmax weights (bf16) into the Pr^T operand,
-//                               Eq. 10 from [P | den] and the value tile, the tile's lowest score, the
-//                               row left out of O^T, the running sums of the weights
+//                               Eq. 10 from [P | den] and the value tile, the running sums of the weights,
+//                               and per row quadrant (a pair of warps) the lowest-scored pair so far
 //   warp 16, one thread         issues [U | Z] = K [W | Q^T] and [P | den] = phi [H | s]; key-tile loads
 //   warp 17, one thread         issues O^T += V^T Pr^T; value-tile loads
 //
@@ -14,6 +14,13 @@
 // tensor memory, so while the score group is busy with tile t the feature group already works on
 // tile t + 1 and the tensor core on the products between them.  Every hand-over is an mbarrier; every
 // wait is bounded, and a wait that runs out raises the block's abort word (bit 8 of the status word).
+//
+// The pair to fold is only known after the last tile.  Every row is therefore attended by the O^T products;
+// each quadrant keeps (q.k, stabiliser, value row, feature row) of its lowest-scored pair, and the epilogue
+// takes the overall lowest out of O^T and the weight sums again (its bf16 weight times its bf16 value row is
+// exact in fp32, so what is subtracted is what the product added, up to the rounding of the running sum).
+// The score group's warps only meet their quadrant partner inside a tile (a 64-thread barrier); a slow warp
+// holds up its partner and the hand-over to the O^T product, not the other quadrants.
 #pragma once
 #include "lola_decode_tc.cuh"
 
@@ -21,6 +28,13 @@ namespace lola {
 
 constexpr int kDec2MaxTiles = 8;
 constexpr int kDec2Threads = 576;      // 16 compute warps + 2 issuing warps
+constexpr float kDec2Lazy = 8.0f;      // log2 units the running maximum may lag behind before O^T is rescaled
+
+__device__ __forceinline__ int ld_global_i32(const int* p) {
+  int v;
+  asm volatile("ld.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
 struct Decode2Misc {
   float qf[kDecQ][128];          // query rows, fp32
@@ -34,16 +48,16 @@ struct Decode2Misc {
   float redmax[2][4][kDecQ];
   float m_s[1][kDecQ];           // running maxima after the last tile (log2 units)
   float z_s[2][kDecQ][128];      // q.k of the tile's rows (log2 units)
-  unsigned long long redkey[4];
-  float red12[4][2];
-  float ssp[128];                // partial squared errors of the second half of the value columns
+  float ssp[2][128];             // partial squared errors of the second half of the value columns (by tile parity)
   float l_s[4][kDecQ];
-  unsigned long long cand_key[kDec2MaxTiles];
-  float cand_score[kDec2MaxTiles], cand_min2[kDec2MaxTiles];
-  int cand_row[kDec2MaxTiles];
-  float cand_z[kDec2MaxTiles][kDecQ];
-  uint4 cand_v[kDec2MaxTiles][16];    // value row, bf16
-  uint4 cand_phi[kDec2MaxTiles][16];  // feature row, bf16
+  // the lowest-scored pair each of the four row quadrants has seen (its warp keeps the key in registers)
+  unsigned long long wb_key[4];
+  float wb_a1[4], wb_a2[4];      // the two lowest scores of the quadrant
+  int wb_row[4];
+  float wb_z[4][kDecQ];          // q.k of that row (log2 units) ...
+  float wb_m[4][kDecQ];          // ... and the stabiliser its weights were taken at
+  uint4 wb_v[4][16];             // value row, bf16
+  uint4 wb_phi[4][16];           // feature row, bf16
   uint64_t bars[20];
   uint32_t tmem_slot;
   int abort_word;
@@ -206,7 +220,6 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       X.knew[tid - 256] = pre_k;
       X.vnew[tid - 256] = pre_v;
     }
-    if (tid < kDec2MaxTiles) { X.cand_key[tid] = ~0ull; X.cand_score[tid] = CUDART_INF_F; X.cand_min2[tid] = CUDART_INF_F; X.cand_row[tid] = 0; }
     // zero phi(Q) and both Pr^T tiles
     for (int i = tid; i < 256; i += 512) {
       *reinterpret_cast<uint4*>(sm + S::phiq + i * 16) = make_uint4(0, 0, 0, 0);
@@ -430,17 +443,24 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     // running maxima of q.k per query row (log2 units; every valid row counts, also the one that will be
     // folded: any m >= the true maximum leaves Eq. 14 unchanged) and this thread's share of the sums
     float lpart[QH], m_run[QR];
+    unsigned long long w_key = ~0ull;                // lowest (score, then youngest) pair of this warp's rows so far
+    float w_a1 = CUDART_INF_F, w_a2 = CUDART_INF_F;  // the two lowest scores of this warp's rows so far
 #pragma unroll
     for (int r = 0; r < QR; ++r) m_run[r] = 0.f;
 #pragma unroll
     for (int r = 0; r < QH; ++r) lpart[r] = 0.f;
+    // token position of this thread's row, fetched one tile ahead (its round trip to the L2 would otherwise sit
+    // in front of the lowest-score reduction of every tile)
+    const int* gpos_u = L.gpos + (size_t)unit * lam;
+    int pos_next = t < lam ? ld_global_i32(gpos_u + t) : pos_ev;
     for (int tile = 0; tile < NT; ++tile) {
       const int i = tile & 1;
       const int R = tile * 128 + t;
       const bool is_g = R < lam;
       const int slot = R - lam;
       const bool scored = is_g || slot == s_ev;
-      const int pos = is_g ? L.gpos[(size_t)unit * lam + R] : pos_ev;
+      const int pos = pos_next;
+      pos_next = (tile + 1 < NT && R + 128 < lam) ? ld_global_i32(gpos_u + R + 128) : pos_ev;
       const uint8_t* vtile = sm + S::stage0 + (size_t)i * S::stage_bytes + S::st_v;
       uint8_t* ptile = sm + stage_pt(i);
 
@@ -461,9 +481,12 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         for (int r = 0; r < QR; ++r) {
           m_new[r] = fmaxf(fmaxf(m_run[r], fmaxf(X.redmax[i][0][r], X.redmax[i][1][r])),
                            fmaxf(X.redmax[i][2][r], X.redmax[i][3][r]));
-          moved = moved || (m_new[r] != m_run[r]);
+          moved = moved || (m_new[r] > m_run[r] + kDec2Lazy);
         }
-        if (moved) {                                 // uniform over the group and rare after the first tiles
+        // The stabiliser only follows the maximum when it has run away by more than 2^kDec2Lazy: any m within
+        // that distance of the true maximum leaves Eq. 14 unchanged (weights up to 2^kDec2Lazy are exact in
+        // bf16's and fp32's range), and moving it means waiting for the O^T product of the tile before.
+        if (moved) {                                 // uniform over the group, rare
           float alpha[QR];
 #pragma unroll
           for (int r = 0; r < QR; ++r) alpha[r] = tc::fast_exp2(m_run[r] - m_new[r]);
@@ -479,9 +502,10 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
             for (int r = 0; r < QR; ++r) ov[r] *= alpha[r];
             tc::tmem_st8(tm_o + lane_addr, ov);
           }
-        }
+          // all rows move together
 #pragma unroll
-        for (int r = 0; r < QR; ++r) m_run[r] = m_new[r];
+          for (int r = 0; r < QR; ++r) m_run[r] = m_new[r];
+        }
 #pragma unroll
         for (int r = 0; r < QH; ++r) {
           const int rr = hf * QH + r;
@@ -492,7 +516,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
       }
       // ---- Eq. 10: this thread's half of the value columns
-      float score;
+      float ss;
       {
         float dn[2];
         tc::tmem_ld2(tm_p + lane_addr + d, dn);
@@ -526,80 +550,60 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         float a0, a1, a2, a3;
         tc::unpack_f2(accA, a0, a1);
         tc::unpack_f2(accB, a2, a3);
-        const float ss = (a0 + a1) + (a2 + a3);
-        if (hf == 1) X.ssp[t] = ss;
-        tc::named_bar_sync(2, 256);
-        score = sqrtf(ss + X.ssp[t]);           // hf = 1 threads double their own half; they do not use the score
+        ss = (a0 + a1) + (a2 + a3);
       }
-      // lowest score of the tile (ties: the younger pair), and the two lowest values
-      unsigned long long key = ~0ull;
+      // every row stays in O^T and in the sums; the one pair that is folded in the end is taken out again
+      // after the last tile, so nothing here needs the other quadrants
+#pragma unroll
+      for (int r = 0; r < QH; ++r) lpart[r] += pw[r];
+      if (hf == 1) X.ssp[i][t] = ss;
+      tc::named_bar_sync(4 + wq, 64);                // the two warps of this row quadrant
       if (hf == 0) {
+        const float score = sqrtf(ss + X.ssp[i][t]);
         if (scored && ok) scu[is_g ? R : lam] = score;
-        if (scored) key = ((unsigned long long)__float_as_uint(score) << 32) | (unsigned)(0x7fffffff - pos);
+        // lowest score of the quadrant's rows in this tile (ties: the younger pair) and the runner-up;
         // scores are norms (>= 0): their bit patterns order like unsigned integers
         const unsigned sb = scored ? __float_as_uint(score) : 0xffffffffu;
         const unsigned smin = __reduce_min_sync(0xffffffffu, sb);
         const unsigned tb_ = (sb == smin && scored) ? (unsigned)(0x7fffffff - pos) : 0xffffffffu;
         const unsigned tmin = __reduce_min_sync(0xffffffffu, tb_);
-        const unsigned long long k = scored || smin != 0xffffffffu ? (((unsigned long long)smin << 32) | tmin) : ~0ull;
         const bool is_min = scored && sb == smin && tb_ == tmin;
         const unsigned s2 = __reduce_min_sync(0xffffffffu, is_min ? 0xffffffffu : sb);
-        const float a1 = smin == 0xffffffffu ? CUDART_INF_F : __uint_as_float(smin);
-        const float a2 = s2 == 0xffffffffu ? CUDART_INF_F : __uint_as_float(s2);
-        if (lane == 0) { X.redkey[wq] = k; X.red12[wq][0] = a1; X.red12[wq][1] = a2; }
-      }
-      tc::named_bar_sync(2, 256);
-      unsigned long long tkey = X.redkey[0];
+        const float c1 = smin == 0xffffffffu ? CUDART_INF_F : __uint_as_float(smin);
+        const float c2 = s2 == 0xffffffffu ? CUDART_INF_F : __uint_as_float(s2);
+        w_a2 = fminf(fmaxf(w_a1, c1), fminf(w_a2, c2));
+        w_a1 = fminf(w_a1, c1);
+        const unsigned long long k = smin != 0xffffffffu ? (((unsigned long long)smin << 32) | tmin) : ~0ull;
+        if (k < w_key) {                             // (uniform over the warp) a new lowest pair of this quadrant:
+          w_key = k;                                 // keep what the fold and Eq. 14 need of it
+          const int src = __ffs(__ballot_sync(0xffffffffu, is_min)) - 1;
+          uint32_t pr[32];
 #pragma unroll
-      for (int w = 1; w < 4; ++w) tkey = X.redkey[w] < tkey ? X.redkey[w] : tkey;
-      // the row left out of O^T: both threads of the row know it from the row's position
-      const unsigned long long rowkey_lo = (unsigned)(0x7fffffff - pos);
-      const bool left_out = scored && (unsigned)tkey == (unsigned)rowkey_lo && tkey != ~0ull;
-      if (left_out) {
-        if (hf == 0) {
-          float a1 = X.red12[0][0], a2 = X.red12[0][1];
+          for (int half = 0; half < 2; ++half) {     // its feature row, read back from tensor memory
+            tc::tmem_ld32u(tm_phi(i) + lane_addr + half * 32, pr);
+            if (is_min) {
+              uint4* dst = &X.wb_phi[wq][half * 8];
 #pragma unroll
-          for (int w = 1; w < 4; ++w) {
-            float b1 = X.red12[w][0], b2 = X.red12[w][1];
-            float lo = fminf(a1, b1), hi = fmaxf(a1, b1);
-            a2 = fminf(hi, fminf(a2, b2));
-            a1 = lo;
+              for (int q = 0; q < 8; ++q) dst[q] = make_uint4(pr[4 * q], pr[4 * q + 1], pr[4 * q + 2], pr[4 * q + 3]);
+            }
           }
-          X.cand_key[tile] = key;
-          X.cand_score[tile] = score;
-          X.cand_min2[tile] = a2;
-          X.cand_row[tile] = R;
+          if (lane < d / 8)                          // its value row: one 16-byte piece per lane
+            X.wb_v[wq][lane] = *reinterpret_cast<const uint4*>(vtile + (lane >> 3) * 16384 + tc::sw128_off(wq * 32 + src, lane & 7));
+          if (is_min) {
+            X.wb_row[wq] = R;
 #pragma unroll
-          for (int r = 0; r < QR; ++r) X.cand_z[tile][r] = X.z_s[i][r][t];
-        } else {
-#pragma unroll
-          for (int ch = 0; ch < d / 8; ++ch)
-            X.cand_v[tile][ch] = *reinterpret_cast<const uint4*>(vtile + (ch >> 3) * 16384 + tc::sw128_off(t, ch & 7));
-        }
-      }
-      if (__any_sync(0xffffffffu, left_out)) {       // its feature row, read back from tensor memory (this thread's half)
-        uint32_t pr[32];
-        tc::tmem_ld32u(tm_phi(i) + lane_addr + hf * 32, pr);
-        if (left_out) {
-          uint32_t* dst = reinterpret_cast<uint32_t*>(&X.cand_phi[tile][0]) + hf * 32;
-#pragma unroll
-          for (int q = 0; q < 32; ++q) dst[q] = pr[q];
-        }
-      }
-      // sums of the weights (the row left out takes its weights back)
-#pragma unroll
-      for (int r = 0; r < QH; ++r) {
-        if (left_out) {
-          const int rr = hf * QH + r;
-          *reinterpret_cast<unsigned short*>(ptile + (t >> 6) * 2048 + tc::sw128_off(rr, (t & 63) >> 3) + (t & 7) * 2) = 0;
-        } else {
-          lpart[r] += pw[r];
+            for (int r = 0; r < QR; ++r) {
+              X.wb_z[wq][r] = X.z_s[i][r][t];
+              X.wb_m[wq][r] = m_run[r];
+            }
+          }
         }
       }
       tc::fence_async_smem();
       tc::fence_before_sync();
       tc::mbar_arrive(bar_ptready(i));
     }
+    if (hf == 0 && lane == 0) { X.wb_key[wq] = w_key; X.wb_a1[wq] = w_a1; X.wb_a2[wq] = w_a2; }
 #pragma unroll
     for (int r = 0; r < QH; ++r) {
       float ls = warp_sum(lpart[r]);
@@ -626,12 +630,13 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   // ---- the pair to fold: lowest (score, then youngest) over the tiles' left-out rows
   int lt = 0;
   {
-    unsigned long long best = X.cand_key[0];
-    for (int i = 1; i < NT; ++i)
-      if (X.cand_key[i] < best) { best = X.cand_key[i]; lt = i; }
+    unsigned long long best = X.wb_key[0];
+#pragma unroll
+    for (int i = 1; i < 4; ++i)
+      if (X.wb_key[i] < best) { best = X.wb_key[i]; lt = i; }
   }
-  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_phi[lt][0]);
-  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[lt][0]);
+  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.wb_phi[lt][0]);
+  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.wb_v[lt][0]);
   if (warp < g) {                                 // phi(q) . phi_fold
     const int r = warp;
     float a = 0.f;
@@ -674,19 +679,17 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       float l0 = 0.f;
 #pragma unroll
       for (int w = 0; w < 4; ++w) l0 += X.l_s[w][r];
-      float num = a0 * opart[cc * QR + r];
-      float den = a0 * l0;
-      for (int ti = 0; ti < NT; ++ti) {
-        if (ti == lt || X.cand_key[ti] == ~0ull) continue;
-        const float p = round_bf16f(tc::fast_exp2(X.cand_z[ti][r] - mf));
-        num = fmaf(p, __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(&X.cand_v[ti][0])[cc]), num);
-        den += p;
-      }
+      // the folded pair leaves the softmax part again: its weight as the tile's product used it (bf16, taken
+      // at the stabiliser of that tile), brought to the final stabiliser like everything else in O^T
+      const float vLc = __bfloat162float(vL[cc]);
+      const float pL = round_bf16f(tc::fast_exp2(X.wb_z[lt][r] - X.wb_m[lt][r])) * tc::fast_exp2(X.wb_m[lt][r] - m0);
+      float num = a0 * fmaf(-pL, vLc, opart[cc * QR + r]);
+      float den = a0 * (l0 - pL);
       const float pn = tc::fast_exp2(X.zn[r] - mf);
       num = fmaf(pn, X.vnew[cc], num);
       den += pn;
       const float e = tc::fast_exp2(-mf);
-      num = fmaf(e * X.dotL[r], __bfloat162float(vL[cc]), num);
+      num = fmaf(e * X.dotL[r], vLc, num);
       den = fmaf(e, X.lden[r] + X.dotL[r], den);
       ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
     }
@@ -694,7 +697,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
 
   // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself) and
   // the new pair enters the window ring; both were fetched at the start
-  const int rowL = X.cand_row[lt];
+  const int rowL = X.wb_row[lt];
   if (okb) {
     constexpr int nch = d / 8;
     if (tid < 2 * nch && rowL < lam) {
@@ -712,11 +715,12 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
     if (tid == 96) {
       // lowest kept / highest folded score of this update
-      float second = X.cand_min2[lt];
-      for (int i = 0; i < NT; ++i)
-        if (i != lt) second = fminf(second, X.cand_score[i]);
+      float second = X.wb_a2[lt];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (i != lt) second = fminf(second, X.wb_a1[i]);
       L.thr[(size_t)unit * 2 + 0] = second;
-      L.thr[(size_t)unit * 2 + 1] = X.cand_score[lt];
+      L.thr[(size_t)unit * 2 + 1] = X.wb_a1[lt];
     }
   }
   if (!okb && tid == 0) atomicOr(L.status, 8);
