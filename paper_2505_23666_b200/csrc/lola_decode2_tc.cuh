@@ -7,8 +7,9 @@
 //   score group   (warps 8-15)  per tile: running maxima and softmax weights (bf16) into the Pr^T operand,
 //                               Eq. 10 from [P | den] and the value tile, the running sums of the weights,
 //                               and per row quadrant (a pair of warps) the lowest-scored pair so far
-//   warp 16, one thread         issues [U | Z] = K [W | Q^T] and [P | den] = phi [H | s]; key-tile loads
+//   warp 16, one thread         issues [P | den] = phi [H | s] (and the linear term H^T phi(Q)^T once)
 //   warp 17, one thread         issues O^T += V^T Pr^T; value-tile loads
+//   warp 18, one thread         issues [U | Z] = K [W | Q^T]; key-tile loads
 //
 // The two groups work on different tiles at the same time: [U | Z] and phi are double-buffered in
 // tensor memory, so while the score group is busy with tile t the feature group already works on
@@ -27,7 +28,7 @@
 namespace lola {
 
 constexpr int kDec2MaxTiles = 8;
-constexpr int kDec2Threads = 576;      // 16 compute warps + 2 issuing warps
+constexpr int kDec2Threads = 608;      // 16 compute warps + 3 issuing warps
 constexpr float kDec2Lazy = 8.0f;      // log2 units the running maximum may lag behind before O^T is rescaled
 
 __device__ __forceinline__ int ld_global_i32(const int* p) {
@@ -105,7 +106,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
 
   const int unit = blockIdx.x, b = unit / L.Hkv, h = unit % L.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int role = warp < 8 ? 0 : (warp < 16 ? 1 : warp - 14);   // 0 feature, 1 score, 2 / 3 issuing threads
+  const int role = warp < 8 ? 0 : (warp < 16 ? 1 : warp - 14);   // 0 feature, 1 score, 2 / 3 / 4 issuing threads
   const int gtid = tid & 255;                // index inside a compute group
   const int gw = warp & 7;
   const int wq = gw & 3;                     // tensor-memory lane quadrant of this warp (= warp % 4)
@@ -127,7 +128,8 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   const uint32_t bar_p = bars + 64u, bar_pfree = bars + 72u;
   auto bar_ptready = [&](int i) { return bars + 80u + 8u * (uint32_t)i; };
   auto bar_o = [&](int i) { return bars + 96u + 8u * (uint32_t)i; };
-  const uint32_t bar_w = bars + 112u, bar_h = bars + 120u, bar_ht = bars + 128u;
+  const uint32_t bar_w = bars + 112u, bar_phiq = bars + 120u, bar_ht = bars + 128u;
+  auto bar_uread = [&](int i) { return bars + 136u + 8u * (uint32_t)i; };
   auto stage_k = [&](int i) { return sbase + S::stage0 + (uint32_t)i * S::stage_bytes + S::st_k; };
   auto stage_v = [&](int i) { return sbase + S::stage0 + (uint32_t)i * S::stage_bytes + S::st_v; };
   auto stage_pt = [&](int i) { return S::stage0 + (uint32_t)i * S::stage_bytes + S::st_pt; };   // offset from sm
@@ -150,12 +152,26 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     pre_k = ldf<T>((const T*)c.k + ((size_t)b * L.Hkv + h) * d + (tid - 256));
     pre_v = ldf<T>((const T*)c.v + ((size_t)b * L.Hkv + h) * d + (tid - 256));
   }
+  // H (fp32 [D][d]) straight into registers: compute thread x gathers, for DPL items (column c, 8 consecutive j),
+  // the eight values H[j][c]; lanes = consecutive columns, so every load of a warp is one 128-byte line.  They
+  // become the bf16 operand image H^T below; no staging buffer, so both stages stream key and value tiles from
+  // the start
+  float pre_h[DPL][8];
+  if (tid < 512) {
+    const float* Hg = L.H + (size_t)unit * D * d;
+#pragma unroll
+    for (int n = 0; n < DPL; ++n) {
+      const int it = tid + 512 * n, cc = it % d, jc = it / d;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) pre_h[n][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+    }
+  }
 
   if (tid == 0) {
     X.abort_word = 0;
-    for (int i = 0; i < 17; ++i) {
-      const bool group = (i == 6 || i == 7 || i == 9 || i == 10 || i == 11 || i == 16);
-      tc::mbar_init(bars + 8u * i, group ? 256u : 1u);
+    for (int i = 0; i < 19; ++i) {
+      const bool group = (i == 6 || i == 7 || i == 9 || i == 10 || i == 11 || i >= 15);
+      tc::mbar_init(bars + 8u * i, i == 16 ? 512u : (group ? 256u : 1u));   // (16: H^T written, by both groups)
     }
     tc::mbar_init_fence();
   }
@@ -166,17 +182,16 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     return;
   }
   if (tid == 17 * 32) {
-    // W^T straight into the operand rows; H (fp32) into the key and value buffers of stage 1, which
-    // the second tile only needs later; the first tile starts to stream at once
+    // W^T straight into the operand rows; the first two tiles start to stream at once
     tc::mbar_expect_tx(bar_w, (uint32_t)kblk * 8192u);
     for (int kb = 0; kb < kblk; ++kb)
       tc::bulk_copy_g2s(sbase + S::b1 + (uint32_t)kb * S::b1_blk, wt_image + ((size_t)h * kblk + kb) * 512, 8192u, bar_w);
     decode2_issue_tile<DPL>(stage_k(0), &tm_gk, &tm_wk, 0, nGB, nRB, unit, bar_kfull(0));
-    const float* Hg = L.H + (size_t)unit * D * d;
-    tc::mbar_expect_tx(bar_h, (uint32_t)(D * d * 4));
-    tc::bulk_copy_g2s(stage_k(1), Hg, 64u * d * 4u, bar_h);
-    tc::bulk_copy_g2s(stage_v(1), Hg + 64 * d, 64u * d * 4u, bar_h);
     decode2_issue_tile<DPL>(stage_v(0), &tm_gv, &tm_wv, 0, nGB, nRB, unit, bar_vfull(0));
+    if (NT > 1) {
+      decode2_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
+      decode2_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
+    }
   }
 
   // ---- operands that stay for the whole unit (compute warps)
@@ -242,73 +257,73 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   const uint32_t idesc3 = tc::make_idesc_bf16(128, 16, true, false);
   bool ok = true;
 
+  if (role < 2) {
+    // H -> bf16 H^T, K-major: row c, 64 j per 128-byte row, two j blocks (lanes = consecutive columns: no conflicts)
+#pragma unroll
+    for (int n = 0; n < DPL; ++n) {
+      const int it = tid + 512 * n, cc = it % d, jc = it / d;
+      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(pre_h[n]);
+    }
+    tc::fence_async_smem();
+    tc::mbar_arrive(bar_ht);
+  }
+
   if (role == 2) {
-    // =================== products of the feature side, key tiles ===================
+    // =================== [P | den] products ===================
     if (lane == 0) {
-      // operand descriptors: the address field (units of 16 bytes) takes the offset of a K step
+      // operand descriptor: the address field (units of 16 bytes) takes the offset of a K step
+      const uint64_t dht = tc::make_desc_sw128(sbase + S::ht, 16, 1024);
+      for (int tile = 0; tile < NT; ++tile) {
+        const int i = tile & 1;
+        ok = tc::mbar_wait(bar_phidone(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;   // phi(tile) is in tensor memory
+        tc::fence_after_sync();
+        if (tile == 0) {
+          ok = tc::mbar_wait(bar_ht, 0, abw) && ok;                              // H^T is in place
+        } else {
+          ok = tc::mbar_wait(bar_pfree, (uint32_t)(tile - 1) & 1u, abw) && ok;   // [P | den] of the tile before is read
+        }
+        tc::fence_after_sync();
+        const uint32_t tph = tm_phi(i);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ts(tm_p, tph + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
+        tc::mma_commit(bar_p);
+        if (tile == 0) {
+          // O^T starts as the linear term H^T phi(Q)^T, with weight exp(0 - m), m = 0 so far; the first O^T
+          // product waits for it
+          ok = tc::mbar_wait(bar_phiq, 0, abw) && ok;
+          tc::fence_after_sync();
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
+                            tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc0, ks > 0);
+          tc::mma_commit(bar_o(0));
+        }
+      }
+    }
+    __syncwarp();
+  } else if (role == 4) {
+    // =================== [U | Z] products, key tiles ===================
+    if (lane == 0) {
       const uint64_t dk0 = tc::make_desc_sw128(stage_k(0), 16, 1024), dk1 = tc::make_desc_sw128(stage_k(1), 16, 1024);
-      const uint64_t db1 = tc::make_desc_sw128(sbase + S::b1, 16, 1024), dht = tc::make_desc_sw128(sbase + S::ht, 16, 1024);
-      auto issue_mma1 = [&](int tile) {
-        const uint64_t dk = (tile & 1) ? dk1 : dk0;
-        const uint32_t tmu = tm_uz(tile & 1);
+      const uint64_t db1 = tc::make_desc_sw128(sbase + S::b1, 16, 1024);
+      ok = tc::mbar_wait(bar_w, 0, abw) && ok;
+      for (int tile = 0; tile < NT; ++tile) {
+        const int i = tile & 1;
+        ok = tc::mbar_wait(bar_kfull(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+        if (tile >= 2)                               // the feature group has read [U | Z] of tile - 2
+          ok = tc::mbar_wait(bar_uread(i), (uint32_t)((tile - 2) >> 1) & 1u, abw) && ok;
+        tc::fence_after_sync();
+        const uint64_t dk = i ? dk1 : dk0;
+        const uint32_t tmu = tm_uz(i);
 #pragma unroll
         for (int ks = 0; ks < d / 16; ++ks)
           tc::mma_bf16_ss(tmu, dk + (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
                           db1 + (uint64_t)(((ks >> 2) * S::b1_blk + (ks & 3) * 32) >> 4), idesc1, ks > 0);
-        tc::mma_commit(bar_u(tile & 1));
-      };
-      // key tiles: tile x + 2 streams into the buffer of tile x once that tile's first product is complete
-      int next_k = 2;                                  // tiles 0 and 1 are loaded by the prologue
-      int next1 = 0;                                   // next first product to issue
-      ok = tc::mbar_wait(bar_w, 0, abw) && ok;
-      // one copy of every step (iteration -1 only issues the first tile's first product): the code of this
-      // thread shares the instruction cache with the two compute groups
-      for (int tile = -1; tile < NT; ++tile) {
-        const int i = tile & 1;
-        if (tile >= 0) {
-          ok = tc::mbar_wait(bar_phidone(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;   // phi(tile) written, [U | Z] of this tile read
-          tc::fence_after_sync();
-          if (tile == 0) {
-            // H^T is in place: stage 1 is free for the second tile; O^T starts as the linear term
-            // H^T phi(Q)^T, with weight exp(0 - m), m = 0 so far
-            ok = tc::mbar_wait(bar_ht, 0, abw) && ok;
-            tc::fence_after_sync();
-            if (NT > 1) {
-              decode2_issue_tile<DPL>(stage_k(1), &tm_gk, &tm_wk, 1, nGB, nRB, unit, bar_kfull(1));
-              decode2_issue_tile<DPL>(stage_v(1), &tm_gv, &tm_wv, 1, nGB, nRB, unit, bar_vfull(1));
-            }
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks)
-              tc::mma_bf16_ss(tm_o, tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
-                              tc::make_desc_sw128(sbase + S::phiq + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc0, ks > 0);
-            tc::mma_commit(bar_o(0));
-          } else {
-            ok = tc::mbar_wait(bar_pfree, (uint32_t)(tile - 1) & 1u, abw) && ok;   // [P | den] of the tile before is read
-            tc::fence_after_sync();
-          }
-          const uint32_t tph = tm_phi(i);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks)
-            tc::mma_bf16_ts(tm_p, tph + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
-          tc::mma_commit(bar_p);
-        }
-        // first products run two tiles ahead of the feature group: the buffer a tile used is free once its
-        // feature rows are written (seen above)
-        const int upto = tile < 0 ? 0 : min(tile + 2, NT - 1);
-        for (; next1 <= upto; ++next1) {
-          while (next_k <= next1) {                    // (the tile's load must have been issued)
-            ok = tc::mbar_wait(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u, abw) && ok;
-            decode2_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
-            ++next_k;
-          }
-          ok = tc::mbar_wait(bar_kfull(next1 & 1), (uint32_t)(next1 >> 1) & 1u, abw) && ok;
-          tc::fence_after_sync();
-          issue_mma1(next1);
-        }
-        // key tiles whose buffer is free already (the product that read it is complete) start to stream now
-        while (next_k < NT && next_k - 2 < next1 && mbar_test(bar_u(next_k & 1), (uint32_t)((next_k - 2) >> 1) & 1u)) {
-          decode2_issue_tile<DPL>(stage_k(next_k & 1), &tm_gk, &tm_wk, next_k, nGB, nRB, unit, bar_kfull(next_k & 1));
-          ++next_k;
+        tc::mma_commit(bar_u(i));
+        if (tile + 2 < NT) {                         // the tile after next streams into this buffer once the product has read it
+          ok = tc::mbar_wait(bar_u(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+          decode2_issue_tile<DPL>(stage_k(i), &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_kfull(i));
         }
       }
     }
@@ -321,6 +336,7 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       for (int tile = 0; tile < NT; ++tile) {
         const int i = tile & 1;
         ok = tc::mbar_wait(bar_ptready(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
+        if (tile == 0) ok = tc::mbar_wait(bar_o(0), 0, abw) && ok;   // the linear term is in O^T
         tc::fence_after_sync();
         const uint64_t dv = i ? dv1 : dv0, dp = i ? dp1 : dp0;
 #pragma unroll
@@ -360,6 +376,8 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       {
         uint32_t u[64];
         tc::tmem_ld64u(tm_uz(i) + lane_addr, u);
+        tc::fence_before_sync();
+        tc::mbar_arrive(bar_uread(i));               // [U | Z] of this tile is in registers: the buffer may take tile + 2
         tc::phi_half(u, hf != 0, exp_kind, pk2);
       }
       if (tile >= 2) {                               // the score group is done with the buffers of tile - 2
@@ -426,19 +444,8 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       zz = warp_sum(zz);
       if (lane == 0) { X.lden[r] = ld; X.zn[r] = zz * sl2; }
     }
-    // H (fp32 [D][d], staged in the buffers of stage 1) -> bf16 H^T, K-major: row c, 64 j per 128-byte row,
-    // two j blocks.  A thread gathers 8 consecutive j of one column c (lanes = consecutive columns: no conflicts).
-    ok = tc::mbar_wait(bar_h, 0, abw) && ok;
-    for (int i = gtid; i < d * (D / 8); i += 256) {
-      const int cc = i % d, jc = i / d;
-      const float* src = reinterpret_cast<const float*>(sm + S::stage0 + S::stage_bytes + ((jc >> 3) ? S::st_v : S::st_k)) + ((jc & 7) * 8) * d + cc;
-      float f8[8];
-#pragma unroll
-      for (int jj = 0; jj < 8; ++jj) f8[jj] = src[jj * d];
-      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
-    }
     tc::fence_async_smem();
-    tc::mbar_arrive(bar_ht);
+    tc::mbar_arrive(bar_phiq);                       // phi(Q) is in its operand rows
 
     // running maxima of q.k per query row (log2 units; every valid row counts, also the one that will be
     // folded: any m >= the true maximum leaves Eq. 14 unchanged) and this thread's share of the sums
@@ -615,118 +622,126 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
   }
 
-  // ---- all products are complete (the thread that issued the last one has seen it complete)
+  // ---- after the last tile the two compute groups split the rest: the feature group folds (Eq. 13), the score
+  // group writes the outputs (Eq. 14) and the memories; the issuing warps go straight to the end
+  if (role < 2) {
+    tc::fence_before_sync();
+    tc::named_bar_sync(9, 512);                      // the score group has finished the last tile
+    tc::fence_after_sync();
+    // the pair to fold: lowest (score, then youngest) over the four quadrants
+    int lt = 0;
+    {
+      unsigned long long best = X.wb_key[0];
+#pragma unroll
+      for (int i = 1; i < 4; ++i)
+        if (X.wb_key[i] < best) { best = X.wb_key[i]; lt = i; }
+    }
+    const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.wb_phi[lt][0]);
+    const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.wb_v[lt][0]);
+    // the stage the last tile did not use is free once the O^T product of the tile before the last is complete
+    const uint32_t free_stage = S::stage0 + (uint32_t)(NT & 1) * S::stage_bytes;
+    if (role == 0) {
+      // ---- Eq. 13: H += phi_fold v_fold^T.  The update (fp32 [D][d], the layout of H) is staged in the free
+      // stage and added to H by bulk reductions: the additions happen at the L2, nothing is read back
+      if (NT >= 2) ok = tc::mbar_wait(bar_o((NT - 1) & 1), (uint32_t)((NT - 1) >> 1) & 1u, abw) && ok;
+      const bool okb = X.abort_word == 0;
+      if (okb) {
+        constexpr int per_row = d / 4;
+        float4* dH = reinterpret_cast<float4*>(sm + free_stage);
+        for (int i = tid; i < D * per_row; i += 256) {
+          const int j = i / per_row, c4 = (i % per_row) * 4;
+          const float pj = __bfloat162float(phiL[j]);
+          const uint2 vv = *reinterpret_cast<const uint2*>(vL + c4);
+          dH[i] = make_float4(pj * bf16lo_f(vv.x), pj * bf16hi_f(vv.x), pj * bf16lo_f(vv.y), pj * bf16hi_f(vv.y));
+        }
+        tc::fence_async_smem();
+      }
+      tc::named_bar_sync(10, 256);
+      if (okb && tid == 0) {
+        float* Hgw = L.H + (size_t)unit * D * d;
+        constexpr uint32_t half_bytes = (uint32_t)(D * d * 4 / 2);
+        tc::bulk_reduce_add_f32(Hgw, sbase + free_stage, half_bytes);
+        tc::bulk_reduce_add_f32(Hgw + D * d / 2, sbase + free_stage + half_bytes, half_bytes);
+        tc::bulk_commit_group();
+      }
+      if (okb && tid < D) atomicAdd(L.s + (size_t)unit * D + tid, __bfloat162float(phiL[tid]));
+    } else {
+      if (gw < g) {                                  // phi(q) . phi_fold
+        const int r = gw;
+        float a = 0.f;
+        for (int j = lane; j < D; j += 32) a = fmaf(X.phiq_f[r][j], __bfloat162float(phiL[j]), a);
+        a = warp_sum(a);
+        if (lane == 0) X.dotL[r] = a;
+      }
+      // O^T is complete with the product of the last tile
+      ok = tc::mbar_wait(bar_o(NT & 1), (uint32_t)(NT >> 1) & 1u, abw) && ok;
+      tc::fence_after_sync();
+      float* opart = reinterpret_cast<float*>(sm + free_stage + S::st_pt);   // [128][QR], in the free stage's Pr^T tile
+      if (gw < 4) {
+        float ov[8];
+        tc::tmem_ld8(tm_o + lane_addr, ov);
+#pragma unroll
+        for (int r = 0; r < QR; ++r) opart[t * QR + r] = ov[r];
+      }
+      tc::named_bar_sync(11, 256);
+      const bool okb = X.abort_word == 0;
+      // ---- Eq. 14: thread (query row r, value column cc)
+      if (okb) {
+        for (int i = gtid; i < g * d; i += 256) {
+          const int r = i / d, cc = i % d;
+          const float m0 = X.m_s[0][r];              // the score group left the final maxima there
+          const float mf = fmaxf(m0, X.zn[r]);
+          const float a0 = tc::fast_exp2(m0 - mf);
+          float l0 = 0.f;
+#pragma unroll
+          for (int w = 0; w < 4; ++w) l0 += X.l_s[w][r];
+          // the folded pair leaves the softmax part again: its weight as the tile's product used it (bf16, taken
+          // at the stabiliser of that tile), brought to the final stabiliser like everything else in O^T
+          const float vLc = __bfloat162float(vL[cc]);
+          const float pL = round_bf16f(tc::fast_exp2(X.wb_z[lt][r] - X.wb_m[lt][r])) * tc::fast_exp2(X.wb_m[lt][r] - m0);
+          float num = a0 * fmaf(-pL, vLc, opart[cc * QR + r]);
+          float den = a0 * (l0 - pL);
+          const float pn = tc::fast_exp2(X.zn[r] - mf);
+          num = fmaf(pn, X.vnew[cc], num);
+          den += pn;
+          const float e = tc::fast_exp2(-mf);
+          num = fmaf(e * X.dotL[r], vLc, num);
+          den = fmaf(e, X.lden[r] + X.dotL[r], den);
+          ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
+        }
+        // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself) and
+        // the new pair enters the window ring; both were fetched at the start
+        const int rowL = X.wb_row[lt];
+        constexpr int nch = d / 8;
+        if (gtid < 2 * nch && rowL < lam) {
+          T* dst = (gtid < nch ? (T*)L.gk : (T*)L.gv) + ((size_t)unit * lam + rowL) * d;
+          *reinterpret_cast<uint4*>(dst + (gtid % nch) * 8) = X.ring_kv[gtid];
+        }
+        if (gtid >= 32 && gtid < 32 + 2 * nch) {
+          const int i = gtid - 32;
+          T* dst = (i < nch ? (T*)L.wk : (T*)L.wv) + ((size_t)unit * eta + s_ev) * d;
+          *reinterpret_cast<uint4*>(dst + (i % nch) * 8) = X.new_kv[i];
+        }
+        if (gtid == 64 && rowL < lam) {
+          L.gpos[(size_t)unit * lam + rowL] = pos_ev;
+          scu[rowL] = scu[lam];
+        }
+        if (gtid == 96) {
+          // lowest kept / highest folded score of this update
+          float second = X.wb_a2[lt];
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (i != lt) second = fminf(second, X.wb_a1[i]);
+          L.thr[(size_t)unit * 2 + 0] = second;
+          L.thr[(size_t)unit * 2 + 1] = X.wb_a1[lt];
+        }
+      }
+    }
+  }
+  if (tid == 0) tc::bulk_wait_group_read();        // the bulk reductions have read shared memory (they are performed by the end of the kernel)
   tc::fence_before_sync();
   __syncthreads();
-  tc::fence_after_sync();
-  const bool okb = X.abort_word == 0;
-  float* opart = reinterpret_cast<float*>(sm + S::stage0 + S::stage_bytes + S::st_v);   // [128][QR], in the free stage 1
-  if (warp < 4) {
-    float ov[8];
-    tc::tmem_ld8(tm_o + lane_addr, ov);
-#pragma unroll
-    for (int r = 0; r < QR; ++r) opart[t * QR + r] = ov[r];
-  }
-  // ---- the pair to fold: lowest (score, then youngest) over the tiles' left-out rows
-  int lt = 0;
-  {
-    unsigned long long best = X.wb_key[0];
-#pragma unroll
-    for (int i = 1; i < 4; ++i)
-      if (X.wb_key[i] < best) { best = X.wb_key[i]; lt = i; }
-  }
-  const __nv_bfloat16* phiL = reinterpret_cast<const __nv_bfloat16*>(&X.wb_phi[lt][0]);
-  const __nv_bfloat16* vL = reinterpret_cast<const __nv_bfloat16*>(&X.wb_v[lt][0]);
-  if (warp < g) {                                 // phi(q) . phi_fold
-    const int r = warp;
-    float a = 0.f;
-    for (int j = lane; j < D; j += 32) a = fmaf(X.phiq_f[r][j], __bfloat162float(phiL[j]), a);
-    a = warp_sum(a);
-    if (lane == 0) X.dotL[r] = a;
-  }
-  // ---- Eq. 13: H += phi_fold v_fold^T.  The update (fp32 [D][d], the layout of H) is staged in the free
-  // buffers of stage 0 and added to H by bulk reductions: the additions happen at the L2, nothing is read back
-  if (okb) {
-    constexpr int per_row = d / 4;
-    float4* dH = reinterpret_cast<float4*>(sm + S::stage0);
-    for (int i = tid; i < D * per_row; i += kDec2Threads) {
-      const int j = i / per_row, c4 = (i % per_row) * 4;
-      const float pj = __bfloat162float(phiL[j]);
-      const uint2 vv = *reinterpret_cast<const uint2*>(vL + c4);
-      dH[i] = make_float4(pj * bf16lo_f(vv.x), pj * bf16hi_f(vv.x), pj * bf16lo_f(vv.y), pj * bf16hi_f(vv.y));
-    }
-    tc::fence_async_smem();
-  }
-  tc::fence_before_sync();
-  __syncthreads();
-  if (okb && tid == 0) {
-    float* Hgw = L.H + (size_t)unit * D * d;
-    constexpr uint32_t half_bytes = (uint32_t)(D * d * 4 / 2);
-    tc::bulk_reduce_add_f32(Hgw, sbase + S::stage0, half_bytes);
-    tc::bulk_reduce_add_f32(Hgw + D * d / 2, sbase + S::stage0 + half_bytes, half_bytes);
-    tc::bulk_commit_group();
-  }
-  if (okb && tid < D) atomicAdd(L.s + (size_t)unit * D + tid, __bfloat162float(phiL[tid]));
-
-  // ---- Eq. 14: thread (query row r, value column cc)
-  if (okb) {
-    const int il = 0;                                // the score group left the final maxima there
-    for (int i = tid; i < g * d; i += kDec2Threads) {
-      const int r = i / d, cc = i % d;
-      const float m0 = X.m_s[il][r];
-      const float mf = fmaxf(m0, X.zn[r]);
-      const float a0 = tc::fast_exp2(m0 - mf);
-      float l0 = 0.f;
-#pragma unroll
-      for (int w = 0; w < 4; ++w) l0 += X.l_s[w][r];
-      // the folded pair leaves the softmax part again: its weight as the tile's product used it (bf16, taken
-      // at the stabiliser of that tile), brought to the final stabiliser like everything else in O^T
-      const float vLc = __bfloat162float(vL[cc]);
-      const float pL = round_bf16f(tc::fast_exp2(X.wb_z[lt][r] - X.wb_m[lt][r])) * tc::fast_exp2(X.wb_m[lt][r] - m0);
-      float num = a0 * fmaf(-pL, vLc, opart[cc * QR + r]);
-      float den = a0 * (l0 - pL);
-      const float pn = tc::fast_exp2(X.zn[r] - mf);
-      num = fmaf(pn, X.vnew[cc], num);
-      den += pn;
-      const float e = tc::fast_exp2(-mf);
-      num = fmaf(e * X.dotL[r], vLc, num);
-      den = fmaf(e, X.lden[r] + X.dotL[r], den);
-      ((T*)c.out)[((size_t)b * L.Hq + h * g + r) * d + cc] = __float2bfloat16_rn(num / den);
-    }
-  }
-
-  // ---- the evicted pair takes the folded member's slot (nothing moves when it is folded itself) and
-  // the new pair enters the window ring; both were fetched at the start
-  const int rowL = X.wb_row[lt];
-  if (okb) {
-    constexpr int nch = d / 8;
-    if (tid < 2 * nch && rowL < lam) {
-      T* dst = (tid < nch ? (T*)L.gk : (T*)L.gv) + ((size_t)unit * lam + rowL) * d;
-      *reinterpret_cast<uint4*>(dst + (tid % nch) * 8) = X.ring_kv[tid];
-    }
-    if (tid >= 32 && tid < 32 + 2 * nch) {
-      const int i = tid - 32;
-      T* dst = (i < nch ? (T*)L.wk : (T*)L.wv) + ((size_t)unit * eta + s_ev) * d;
-      *reinterpret_cast<uint4*>(dst + (i % nch) * 8) = X.new_kv[i];
-    }
-    if (tid == 64 && rowL < lam) {
-      L.gpos[(size_t)unit * lam + rowL] = pos_ev;
-      scu[rowL] = scu[lam];
-    }
-    if (tid == 96) {
-      // lowest kept / highest folded score of this update
-      float second = X.wb_a2[lt];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (i != lt) second = fminf(second, X.wb_a1[i]);
-      L.thr[(size_t)unit * 2 + 0] = second;
-      L.thr[(size_t)unit * 2 + 1] = X.wb_a1[lt];
-    }
-  }
-  if (!okb && tid == 0) atomicOr(L.status, 8);
-  if (tid == 0) tc::bulk_wait_group_all();         // the bulk reductions have read shared memory and are performed
-  tc::fence_before_sync();
-  __syncthreads();
+  if (tid == 0 && X.abort_word != 0) atomicOr(L.status, 8);
   if (warp == 0) tc::tmem_dealloc(tmem, 512);
 }
 
