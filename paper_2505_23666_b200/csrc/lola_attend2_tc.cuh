@@ -11,10 +11,11 @@
 //                    exp(z - m) rounded to bf16 and written back over S as the A operand of PV
 //   warp 16          issues every tcgen05.mma:  S_w = Q_w K^T,  O_w += P_w V  (P_w in tensor memory)
 //   warp 17          TMA producer
-// After the last tile the feature map of the queries is computed (U_w = Q_w W on the tensor cores, one
-// thread per row), scaled by exp(-m) and fed as a tensor-memory A operand into O_w += phi H (H from its
-// bf16 operand image, bulk-copied at the start), so the linear term lands in the same accumulator; its
-// normaliser exp(-m) phi . s is added to the row's denominator.
+// Before the first tile the feature map of the queries is computed (U_w = Q_w W on the tensor cores into the
+// score columns, two threads per row) and fed as a tensor-memory A operand into O_w = phi H (H from its bf16
+// operand image, bulk-copied at the start): the linear term is the first thing in the accumulator, with the
+// weight exp(0 - m) of a key whose score is 0 (m = 0 at that point), and follows the stabiliser like every
+// other summand; its normaliser phi . s starts the row's denominator.  This runs while the first tiles load.
 // Every wait on an mbarrier is bounded; a wait that runs out sets bit 64 of the status word and makes
 // the other waits of the CTA return at once.
 #pragma once
@@ -109,6 +110,8 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   tc::grid_dep_wait();                               // everything before this kernel in the stream is complete
   if (tid == 0 && before_scoring) tc::grid_dep_launch_dependents();
   const uint32_t tmem = X.tmem_slot;
+  if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
+  __syncthreads();
 
   // block `blk` of the key stream -> TMA source
   auto issue_block = [&](uint32_t dst, int blk, bool is_v, uint32_t bar) {
@@ -138,10 +141,14 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
             tc::tma_load_4d(sbase + S::q + (uint32_t)w * 32768u + (uint32_t)cb * 16384u + (uint32_t)hs * 8192u, &tm_q, cb * 64, head,
                             0, b, BAR(A2_QFULL));
         }
+      // W^T image into the key buffer of stage 1, which the second tile takes over once U = Q W has read it
+      tc::mbar_expect_tx(BAR(A2_WFULL), (uint32_t)kblk * 8192u);
+      tc::bulk_copy_g2s(sbase + S::stage0 + S::stage_bytes + S::st_k, wt_image + (size_t)h * kblk * 512, kblk * 8192u, BAR(A2_WFULL));
       for (int kt = 0; kt < NT; ++kt) {
         const int st = kt & 1;
         const uint32_t stage = sbase + S::stage0 + (uint32_t)st * S::stage_bytes;
-        if (kt >= 2) ok = WAIT(A2_KEMPTY + st, ((kt >> 1) - 1) & 1) && ok;
+        if (st == 1) ok = WAIT(A2_KEMPTY + 1, (kt >> 1) & 1) && ok;   // (its first completion is the read of W^T)
+        else if (kt >= 2) ok = WAIT(A2_KEMPTY + 0, ((kt >> 1) - 1) & 1) && ok;
         tc::mbar_expect_tx(BAR(A2_KFULL + st), (uint32_t)kblk * 16384u);
         issue_block(stage + S::st_k, 2 * kt, false, BAR(A2_KFULL + st));
         issue_block(stage + S::st_k + 8192u, 2 * kt + 1, false, BAR(A2_KFULL + st));
@@ -149,15 +156,6 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         tc::mbar_expect_tx(BAR(A2_VFULL + st), (uint32_t)kblk * 16384u);
         issue_block(stage + S::st_v, 2 * kt, true, BAR(A2_VFULL + st));
         issue_block(stage + S::st_v + 8192u, 2 * kt + 1, true, BAR(A2_VFULL + st));
-      }
-      // W^T image into the key buffer of the stage the last tile does not use
-      {
-        const int so = NT & 1;                                    // stage of tile NT - 2 (or the unused one)
-        const int uses = (NT - so + 1) / 2;                       // tiles that went through stage `so`
-        if (uses >= 1) ok = WAIT(A2_KEMPTY + so, (uses - 1) & 1) && ok;
-        tc::mbar_expect_tx(BAR(A2_WFULL), (uint32_t)kblk * 8192u);
-        tc::bulk_copy_g2s(sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k, wt_image + (size_t)h * kblk * 512, kblk * 8192u,
-                      BAR(A2_WFULL));
       }
       if (!ok) atomicOr(L.status, 64);
     }
@@ -185,56 +183,54 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       auto issue_pv = [&](int w, int kt) {
         const uint64_t dv = (kt & 1) ? dv1 : dv0;
         const uint32_t to = tmem + 256u + (uint32_t)w * 128u, tp = tmem + (uint32_t)w * 128u;
-        const uint32_t acc0 = kt > 0 ? 1u : 0u;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          tc::mma_bf16_ts(to, tp + (uint32_t)(ks >> 2) * 64u + (ks & 3) * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, ks > 0 ? 1u : acc0);
+        for (int ks = 0; ks < 8; ++ks)                                   // (the linear term is in O_w already)
+          tc::mma_bf16_ts(to, tp + (uint32_t)(ks >> 2) * 64u + (ks & 3) * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, 1u);
         tc::mma_commit(BAR(A2_ODONE + w));
       };
+      // ---- linear term first: U_w = Q_w W into the score columns, then O_w = phi(Q_w) H
       ok = WAIT(A2_QFULL, 0) && ok;
-      ok = WAIT(A2_KFULL + 0, 0) && ok;
+      ok = WAIT(A2_WFULL, 0) && ok;
       tc::fence_after_sync();
-      for (int w = 0; w < nw; ++w) issue_s(w, 0);
-      tc::mma_commit(BAR(A2_KEMPTY + 0));
-      const int so = NT & 1;                                             // the W^T image sits in the key buffer of this stage
-      const uint32_t wt = sbase + S::stage0 + (uint32_t)so * S::stage_bytes + S::st_k;
-      for (int kt = 0; kt < NT; ++kt) {
-        const int st = kt & 1;
-        ok = WAIT(A2_VFULL + st, (kt >> 1) & 1) && ok;
-        if (kt + 1 < NT) ok = WAIT(A2_KFULL + (st ^ 1), ((kt + 1) >> 1) & 1) && ok;
+      {
+        const uint32_t wt = sbase + S::stage0 + S::stage_bytes + S::st_k;
         for (int w = 0; w < nw; ++w) {
-          ok = WAIT(A2_PREADY + w, kt & 1) && ok;
-          tc::fence_after_sync();
-          issue_pv(w, kt);
-          if (kt + 1 < NT) {
-            issue_s(w, kt + 1);
-          } else {
-            // after the last PV of this query tile, U = Q W of the linear term goes into its score columns
-            // (the tensor pipe runs in order: the weights there are consumed first)
-            if (w == 0) ok = WAIT(A2_WFULL, 0) && ok;
 #pragma unroll
-            for (int ks = 0; ks < d / 16; ++ks)
-              tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
-                              tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                              tc::make_desc_sw128(wt + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024),
-                              tc::make_idesc_bf16(128, 64, false, false), ks > 0);
-            tc::mma_commit(BAR(A2_SFULL + w));
-          }
+          for (int ks = 0; ks < d / 16; ++ks)
+            tc::mma_bf16_ss(tmem + (uint32_t)w * 128u,
+                            tc::make_desc_sw128(sbase + S::q + (uint32_t)w * 32768u + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                            tc::make_desc_sw128(wt + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024),
+                            tc::make_idesc_bf16(128, 64, false, false), ks > 0);
+          tc::mma_commit(BAR(A2_SFULL + w));                              // completion 0 of S_w: U_w
         }
-        tc::mma_commit(BAR(A2_VEMPTY + st));
-        if (kt + 1 < NT) tc::mma_commit(BAR(A2_KEMPTY + (st ^ 1)));
+        tc::mma_commit(BAR(A2_KEMPTY + 1));                               // W^T is read: the second tile may load
       }
-      // ---- linear term
       ok = WAIT(A2_HFULL, 0) && ok;
+      ok = WAIT(A2_KFULL + 0, 0) && ok;
       for (int w = 0; w < nw; ++w) {
-        ok = WAIT(A2_PREADY + w, NT & 1) && ok;                         // scaled phi(Q_w) in tensor memory
+        ok = WAIT(A2_PREADY + w, 0) && ok;                                // phi(Q_w) in tensor memory
         tc::fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
           tc::mma_bf16_ts(tmem + 256u + (uint32_t)w * 128u, tmem + (uint32_t)w * 128u + 64u + ks * 8,
                           tc::make_desc_sw128(sbase + S::ht + (ks >> 2) * S::ht_blk + (ks & 3) * 32, 16, 1024),
-                          tc::make_idesc_bf16(128, d, false, false), 1u);
-        tc::mma_commit(BAR(A2_ODONE + w));
+                          tc::make_idesc_bf16(128, d, false, false), ks > 0);
+        tc::mma_commit(BAR(A2_ODONE + w));                                // completion 0 of O_w: the linear term
+        issue_s(w, 0);                                                    // (the tensor pipe runs in order: phi is consumed first)
+      }
+      tc::mma_commit(BAR(A2_KEMPTY + 0));
+      for (int kt = 0; kt < NT; ++kt) {
+        const int st = kt & 1;
+        ok = WAIT(A2_VFULL + st, (kt >> 1) & 1) && ok;
+        if (kt + 1 < NT) ok = WAIT(A2_KFULL + (st ^ 1), ((kt + 1) >> 1) & 1) && ok;
+        for (int w = 0; w < nw; ++w) {
+          ok = WAIT(A2_PREADY + w, (kt + 1) & 1) && ok;
+          tc::fence_after_sync();
+          issue_pv(w, kt);
+          if (kt + 1 < NT) issue_s(w, kt + 1);
+        }
+        tc::mma_commit(BAR(A2_VEMPTY + st));
+        if (kt + 1 < NT) tc::mma_commit(BAR(A2_KEMPTY + (st ^ 1)));
       }
       if (!ok) atomicOr(L.status, 64);
     }
@@ -251,8 +247,60 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     const uint32_t tm_sb = tm_s + (uint32_t)hf * 64u;  // this thread's 64 score columns; its weights go to the first 32
     const uint32_t tm_o = tmem + 256u + (uint32_t)w * 128u + lane_addr;
     constexpr int HC = d / 2;
-    if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
-    float m_used = 0.f, l = 0.f;                       // log2 units; m >= 0 is the stabiliser max(0, max z)
+    // ---- linear term first
+    ok = WAIT(A2_SFULL + w, 0) && ok;                  // U = Q W is in the first 64 score columns
+    tc::fence_after_sync();
+    float m_used = 0.f, l;                             // log2 units; m >= 0 is the stabiliser max(0, max z)
+    {
+      // this thread's half of phi(q) (hf = 0: softmax(u), 1: softmax(-u)), with weight exp(0 - m), m = 0: bf16 pairs
+      // into columns 64 + 32 hf .. of S_w (A operand of the linear product)
+      float e[64];
+      tc::tmem_ld64(tm_s, e);
+      const float em = (c.att_flags & 1) ? 0.f : 1.0f;   // (0: the queries do not see H, s)
+      const float sgn = hf ? -kLog2e : kLog2e;
+      float scale;
+      if (L.phi_kind == 1) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
+        scale = em;
+      } else {
+        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) { m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn); }
+        const float mm = fmaxf(m0, m1);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) {
+          e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
+          e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
+        }
+        scale = em / (s0 + s1);
+      }
+      float ld0 = 0.f, ld1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < 64; i += 2) {
+        e[i] *= scale;
+        e[i + 1] *= scale;
+        ld0 = fmaf(e[i], X.s_vec[hf * 64 + i], ld0);
+        ld1 = fmaf(e[i + 1], X.s_vec[hf * 64 + i + 1], ld1);
+      }
+      l = ld0 + ld1;                                   // this half of the normaliser phi . s starts the sum of the weights
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) pk[j >> 1] = pack_bf16x2(e[c0 + j], e[c0 + j + 1]);
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n" ::"r"(
+                tm_s + 64 + hf * 32 + (c0 >> 1)),
+            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]), "r"(pk[8]), "r"(pk[9]),
+            "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
+            : "memory");
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    tc::fence_before_sync();
+    tc::mbar_arrive(BAR(A2_PREADY + w));               // completion 0: phi(Q_w) is in columns 64.. of S_w
     for (int kt = 0; kt < NT; ++kt) {
       // valid leading columns of this thread's 64-key block of the tile, for this row
       const int blk = 2 * kt + hf;
@@ -262,7 +310,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       else if (blk == nGB + nRB) lim = min(n, tok + 1);
       else lim = 0;
       lim = max(0, min(64, lim));
-      ok = WAIT(A2_SFULL + w, kt & 1) && ok;
+      ok = WAIT(A2_SFULL + w, (kt + 1) & 1) && ok;
       tc::fence_after_sync();
       float sv[64];
       tc::tmem_ld64(tm_sb, sv);
@@ -289,8 +337,8 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         const float alpha = tc::fast_exp2(m_used - m_new);
         l *= alpha;
         m_used = m_new;
-        if (kt > 0) {
-          ok = WAIT(A2_ODONE + w, (kt - 1) & 1) && ok;
+        {
+          ok = WAIT(A2_ODONE + w, kt & 1) && ok;         // the product of the tile before (or the linear term) is complete
           tc::fence_after_sync();
 #pragma unroll
           for (int c0 = 0; c0 < HC; c0 += 8) {         // this thread's half of the row's output columns
@@ -331,70 +379,22 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       tc::fence_before_sync();
       tc::mbar_arrive(BAR(A2_PREADY + w));
     }
-    // ---- linear term: once the last PV of this tile has read P_w, S_w may be overwritten
-    ok = WAIT(A2_SFULL + w, NT & 1) && ok;             // U = Q W is there (and every PV of this tile is complete)
-    tc::fence_after_sync();
-    float lden = 0.f;                                  // the other half of the row's denominator
-    {
-      // this thread's half of phi(q) (hf = 0: softmax(u), 1: softmax(-u)), scaled by exp(-m): bf16 pairs
-      // into columns 64 + 32 hf .. of S_w (A operand of the linear product)
-      float e[64];
-      tc::tmem_ld64(tm_s, e);
-      const float em = (c.att_flags & 1) ? 0.f : tc::fast_exp2(-m_used);   // (0: the queries do not see H, s)
-      const float sgn = hf ? -kLog2e : kLog2e;
-      float scale;
-      if (L.phi_kind == 1) {
-#pragma unroll
-        for (int i = 0; i < 64; ++i) e[i] = tc::fast_exp2(e[i] * sgn);
-        scale = em;
-      } else {
-        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
-#pragma unroll
-        for (int i = 0; i < 64; i += 2) { m0 = fmaxf(m0, e[i] * sgn); m1 = fmaxf(m1, e[i + 1] * sgn); }
-        const float mm = fmaxf(m0, m1);
-        float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-        for (int i = 0; i < 64; i += 2) {
-          e[i] = tc::fast_exp2(fmaf(e[i], sgn, -mm)); s0 += e[i];
-          e[i + 1] = tc::fast_exp2(fmaf(e[i + 1], sgn, -mm)); s1 += e[i + 1];
-        }
-        scale = em / (s0 + s1);
-      }
-      float ld0 = 0.f, ld1 = 0.f;
-#pragma unroll
-      for (int i = 0; i < 64; i += 2) {
-        e[i] *= scale;
-        e[i + 1] *= scale;
-        ld0 = fmaf(e[i], X.s_vec[hf * 64 + i], ld0);
-        ld1 = fmaf(e[i + 1], X.s_vec[hf * 64 + i + 1], ld1);
-      }
-      X.hx[w][hf][t] = l + ld0 + ld1;
-      tc::named_bar_sync(1 + w, 256);                  // both halves have read U before columns 64.. are overwritten
-#pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 32) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) pk[j >> 1] = pack_bf16x2(e[c0 + j], e[c0 + j + 1]);
-        asm volatile(
-            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n" ::"r"(
-                tm_s + 64 + hf * 32 + (c0 >> 1)),
-            "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]), "r"(pk[8]), "r"(pk[9]),
-            "r"(pk[10]), "r"(pk[11]), "r"(pk[12]), "r"(pk[13]), "r"(pk[14]), "r"(pk[15])
-            : "memory");
-      }
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-      lden = X.hx[w][hf ^ 1][t];
-    }
-    tc::fence_before_sync();
-    tc::mbar_arrive(BAR(A2_PREADY + w));               // phase NT
+    // ---- the two halves of the row's denominator meet (the extra barrier: the partner has read this row's last
+    // maxima before the slot is reused)
+    tc::named_bar_sync(1 + w, 256);
+    X.hx[w][hf][t] = l;
+    tc::named_bar_sync(1 + w, 256);
+    const float lden = X.hx[w][hf ^ 1][t];
     ok = WAIT(A2_ODONE + w, NT & 1) && ok;
     tc::fence_after_sync();
     {
-      // the tile's outputs are staged in the free value buffer of stage w in the layout of a TMA box
-      // ([head slot][64-column block][64 tokens][128 bytes], 128-byte swizzle) and stored by one thread:
-      // 576 threads storing 16 bytes at a time would take the load/store unit 2 us
+      // the tile's outputs are staged in the layout of a TMA box ([head slot][64-column block][64 tokens]
+      // [128 bytes], 128-byte swizzle) and stored by one thread: 576 threads storing 16 bytes at a time would take
+      // the load/store unit 2 us.  The staging buffers are the key (w = 0) and value (w = 1) buffers of the stage
+      // the last tile did not use: the other query tile's last product may still be reading the last tile
       const float inv = 1.0f / (X.hx[w][hf][t] + lden);
-      uint8_t* stg = sm + S::stage0 + (size_t)w * S::stage_bytes + S::st_v;
+      const uint32_t stg_off = S::stage0 + (uint32_t)(NT & 1) * S::stage_bytes + (w ? S::st_v : S::st_k);
+      uint8_t* stg = sm + stg_off;
       const int hs = t >> 6;
 #pragma unroll
       for (int c0 = 0; c0 < HC; c0 += 32) {
@@ -414,7 +414,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       tc::fence_async_smem();
       tc::named_bar_sync(1 + w, 256);
       if (t == 0 && hf == 0 && ok) {
-        const uint32_t sstg = sbase + S::stage0 + (uint32_t)w * S::stage_bytes + S::st_v;
+        const uint32_t sstg = sbase + stg_off;
         for (int s2 = 0; s2 < 2; ++s2) {
           const int hl2 = (qt0 + w) * 2 + s2;
           if (hl2 >= g) continue;                      // (rows of tokens >= n lie outside the tensor: not written)
