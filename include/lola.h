@@ -267,7 +267,7 @@ enum {
   LOLA_PATH_UPDATE_GENERIC = 1u << 8,
   LOLA_PATH_DECODE_FUSED = 1u << 9,      /* the generation step as one kernel (units of up to 8 row tiles)  */
   LOLA_PATH_DECODE_FUSED_LONG = 1u << 10,/* the same for units of 9 to 16 row tiles                         */
-  LOLA_PATH_H_IMAGE_REBUILD = 1u << 11   /* the tensor-core operand image of H had to be rebuilt first      */
+  LOLA_PATH_H_IMAGE_REBUILD = 1u << 11   /* (never reported: every kernel reads H itself)                   */
 };
 typedef struct lola_call_info {
   uint32_t paths;                        /* OR of LOLA_PATH_*                                               */

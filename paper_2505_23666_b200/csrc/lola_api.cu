@@ -30,7 +30,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct StateLayout {
-  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, himg, wt, total;
+  size_t status, H, s, gk, gv, gpos, score, wk, wv, fold_idx, move_src, move_dst, counts, thr, wt, total;
 };
 
 bool config_ok(const lola_config* c) {
@@ -69,9 +69,7 @@ StateLayout make_layout(const lola_config& c) {
   l.move_dst = take(U * cm * 4);
   l.counts = take(U * 4 * 4);
   l.thr = take(U * 2 * 4);
-  // H of every unit as a bf16 tensor-core operand image, then W^T of every KV head in operand layout
-  // (bf16 layers with F = 64 only)
-  l.himg = take(c.dtype == LOLA_BF16 && c.feat_half == 64 ? U * 2 * d * 64 * 2 : 0);
+  // W^T of every KV head in tensor-core operand layout (bf16 layers with F = 64 only)
   l.wt = take(c.dtype == LOLA_BF16 && c.feat_half == 64 ? (size_t)c.n_kv_heads * d * 64 * 2 : 0);
   l.total = o;
   return l;
@@ -172,7 +170,6 @@ struct lola_state {
   bool fused_decode = false;           // shapes the one-kernel generation step is built for
   int sm_count = 0;                    // SMs of the device (grid of the persistent generation kernel)
   bool have_maps = false;              // TMA descriptors of the sparse cache and the window ring exist
-  bool himg_valid = false;             // the bf16 operand image of H matches H
   // lola_prefill_host: two copy streams and the events that order them against the kernels (made at first use)
   cudaStream_t cp_in = nullptr, cp_out = nullptr;
   cudaEvent_t ev_start = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
@@ -224,16 +221,6 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-template <int DPL>
-int ensure_h_image(lola_state* st, cudaStream_t s) {
-  if (st->himg_valid) return LOLA_OK;
-  LaunchScope scope(st, LOLA_KERNEL_UPDATE, s, LOLA_PATH_H_IMAGE_REBUILD, st->L.B * st->L.Hkv);
-  k_build_ht_image<DPL><<<st->L.B * st->L.Hkv, 256, 0, s>>>(st->L, (__nv_bfloat16*)(st->base + st->lay.himg));
-  if (cudaGetLastError() != cudaSuccess) return LOLA_ERR_CUDA;
-  st->himg_valid = true;
-  return LOLA_OK;
-}
-
 // before_scoring: the kernel after this one in the stream is the scoring kernel of the same call, which only
 // reads the memories and runs beside this one: it is let go once this kernel has seen everything before it
 // complete, and it waits for this kernel at its end (so that whatever follows sees both complete).
@@ -246,12 +233,11 @@ int launch_attend(lola_state* st, const Call& c, cudaStream_t s, bool before_sco
     CUtensorMap tq, tk, tv, tout;
     if (make_tokens_map(&tq, c.q, L.B, c.nq, L.Hq, L.d) && make_tokens_map(&tk, c.k, L.B, c.n, L.Hkv, L.d) &&
         make_tokens_map(&tv, c.v, L.B, c.n, L.Hkv, L.d) && make_tokens_map(&tout, c.out, L.B, c.nq, L.Hq, L.d)) {
-      if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
       dim3 grid2(((L.g + 1) / 2 + 1) / 2, L.B * L.Hkv);
       LaunchScope scope(st, LOLA_KERNEL_ATTEND, s, LOLA_PATH_ATTEND_TMA, (int)(grid2.x * grid2.y));
       const cudaError_t le = launch_pdl(k_attend2_tc<DPL>, grid2, dim3(kAt2Threads), Attend2Smem<DPL>::bytes, s, L, c, st->tm_gk, st->tm_gv,
                                         st->tm_wk, st->tm_wv, tq, tk, tv, tout, (const uint4*)(st->base + st->lay.wt),
-                                        (const __nv_bfloat16*)(st->base + st->lay.himg), before_scoring ? 1 : 0);
+                                        before_scoring ? 1 : 0);
       return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
     }
   }
@@ -290,23 +276,21 @@ int launch_score_select(lola_state* st, const Call& c, cudaStream_t ss, int busy
     if (U * ((NT + t2 - 1) / t2) <= avail) tpc = t2;
   }
   const uint4* img = (const uint4*)(st->base + st->lay.wt);
-  __nv_bfloat16* himg = (__nv_bfloat16*)(st->base + st->lay.himg);
   // the selection (Eq. 12) runs in the scoring kernel: the last block of a unit to finish does it
   dim3 grid((NT + tpc - 1) / tpc, U);
   LaunchScope scope(st, LOLA_KERNEL_SCORE, ss, LOLA_PATH_SCORE_TMA, (int)(grid.x * grid.y));
   const cudaError_t le = launch_pdl(k_score2_tc<DPL>, grid, dim3(kSc2Threads), Score2Smem<DPL>::bytes, ss, L, c, st->tm_gk, st->tm_gv, st->tm_wk,
-                                    st->tm_wv, img, (const __nv_bfloat16*)himg, tpc, busy_sms > 0 ? 1 : 0);
+                                    st->tm_wv, img, tpc, busy_sms > 0 ? 1 : 0);
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
-// Eq. 13 fold, moves into the sparse cache and window roll from the selection's work lists; keeps the
-// operand image of H current.
+// Eq. 13 fold (added to H in memory), moves into the sparse cache and window roll from the selection's work lists.
 template <int DPL>
 int launch_apply(lola_state* st, const Call& c, cudaStream_t s) {
   const Layer& L = st->L;
   LaunchScope scope(st, LOLA_KERNEL_UPDATE, s, LOLA_PATH_APPLY_TMA, L.B * L.Hkv);
   const cudaError_t le = launch_pdl(k_update2_tc<DPL, 2>, dim3(L.B * L.Hkv), dim3(kUp2Threads), Update2Smem<DPL>::bytes, s, L, c,
-                                    (const uint4*)(st->base + st->lay.wt), (__nv_bfloat16*)(st->base + st->lay.himg));
+                                    (const uint4*)(st->base + st->lay.wt), (__nv_bfloat16*)nullptr);
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
 
@@ -317,7 +301,6 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   // chunkwise update on TMA-fed tensor-core kernels: every leaving pair already sits in the ring, the
   // occupied part of the sparse cache is a whole number of 64-slot blocks
   if (fast_update_path(st, c)) {
-    if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
     int rc = launch_score_select<DPL>(st, c, s);
     return rc == LOLA_OK ? launch_apply<DPL>(st, c, s) : rc;
   }
@@ -344,7 +327,6 @@ int launch_update_chain(lola_state* st, const Call& c, cudaStream_t s) {
   if (st->have_maps && !st->force_chain && (c.mode == UPD_NONE || c.mode == UPD_APPEND) && c.r <= kUp2MaxFold)
     return launch_apply<DPL>(st, c, s);  // nothing folds: moves from the work lists and the window roll
   LaunchScope scope(st, LOLA_KERNEL_UPDATE, s, LOLA_PATH_UPDATE_GENERIC, U);
-  if (c.mode == UPD_SELECT || c.mode == UPD_FOLD_ALL) st->himg_valid = false;   // H changes without its operand image
   k_update<T, DPL><<<U, kUpdThreads, update_smem_floats<DPL>(L.D) * 4, s>>>(L, c);
   return cudaGetLastError() == cudaSuccess ? LOLA_OK : LOLA_ERR_CUDA;
 }
@@ -358,7 +340,6 @@ int run_prefill(lola_state* st, Call c, cudaStream_t s) {
   // in its last block per unit) start; the scoring kernel waits for the attention kernel only at its end; the
   // fold waits for the scoring kernel, hence for both.
   if (c.out && fast_update_path(st, c)) {
-    if (ensure_h_image<DPL>(st, s) != LOLA_OK) return LOLA_ERR_CUDA;
     rc = launch_attend<T, DPL>(st, c, s, true);
     if (rc != LOLA_OK) return rc;
     rc = launch_score_select<DPL>(st, c, s, (((st->L.g + 1) / 2 + 1) / 2) * st->L.B * st->L.Hkv);
@@ -398,7 +379,6 @@ int run_decode(lola_state* st, Call c, cudaStream_t s) {
   const bool ablation = (st->cfg.flags & (LOLA_FLAG_QUERY_NO_LINEAR | LOLA_FLAG_QUERY_NO_SPARSE)) != 0;
   if (st->fused_decode && !st->force_chain && !ablation && c.mode == UPD_SELECT && c.r == 1 && c.count_g == st->L.lam)
   {
-    st->himg_valid = false;              // the fused step folds into H only
     return launch_decode_fused<DPL>(st, c, s);
   }
   int rc = launch_update_chain<T, DPL>(st, c, s);
@@ -569,7 +549,6 @@ int lola_reset_state(lola_state* st, void* stream) {
   if (cudaMemsetAsync(L.score, 0xFF, U * ((size_t)c.sparse + c.max_chunk) * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
   if (cudaMemsetAsync(L.thr, 0xFF, U * 2 * 4, s) != cudaSuccess) return LOLA_ERR_CUDA;
   st->n_seen = 0;
-  st->himg_valid = true;               // H = 0 and its operand image = 0
   return LOLA_OK;
 }
 
@@ -832,7 +811,6 @@ int lola_write_state(lola_state* st, const lola_state_view* v, void* stream) {
   ok = ok && cudaMemsetAsync(L.status, 0, 4, s) == cudaSuccess;      // a replaced state starts healthy
   if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return LOLA_ERR_CUDA;   // host staging dies here
   st->n_seen = n_seen;
-  st->himg_valid = false;
   return LOLA_OK;
 }
 
@@ -864,7 +842,6 @@ int lola_set_tokens_seen(lola_state* st, int64_t n_seen) {
   if (!st) return LOLA_ERR_ARG;
   if (n_seen < 0 || n_seen > 0x7fffffffLL) return LOLA_ERR_SHAPE;
   st->n_seen = n_seen;
-  st->himg_valid = false;              // the caller replaced the buffer: rebuild H's operand image when needed
   return LOLA_OK;
 }
 

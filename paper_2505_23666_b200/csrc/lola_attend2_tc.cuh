@@ -13,7 +13,7 @@
 //   warp 17          TMA producer
 // Before the first tile the feature map of the queries is computed (U_w = Q_w W on the tensor cores into the
 // score columns, two threads per row) and fed as a tensor-memory A operand into O_w = phi H (H from its bf16
-// operand image, bulk-copied at the start): the linear term is the first thing in the accumulator, with the
+// operand image, made from H at the start): the linear term is the first thing in the accumulator, with the
 // weight exp(0 - m) of a key whose score is 0 (m = 0 at that point), and follows the stabiliser like every
 // other summand; its normaliser phi . s starts the row's denominator.  This runs while the first tiles load.
 // Every wait on an mbarrier is bounded; a wait that runs out sets bit 64 of the status word and makes
@@ -60,7 +60,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
              const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
              const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_ck,
              const __grid_constant__ CUtensorMap tm_cv, const __grid_constant__ CUtensorMap tm_out, const uint4* wt_image,
-             const __nv_bfloat16* ht_image, int before_scoring) {
+             int before_scoring) {
   using S = Attend2Smem<DPL>;
   constexpr int d = DPL * 32;
   constexpr int kblk = d / 64;
@@ -96,7 +96,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
 
   if (tid == 0) {
     X.abort_word = 0;
-    for (int i = 0; i < 17; ++i) tc::mbar_init(BAR(i), (i == A2_PREADY || i == A2_PREADY + 1) ? 256u : 1u);
+    for (int i = 0; i < 17; ++i) tc::mbar_init(BAR(i), i == A2_HFULL ? 512u : ((i == A2_PREADY || i == A2_PREADY + 1) ? 256u : 1u));
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
@@ -110,8 +110,30 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   tc::grid_dep_wait();                               // everything before this kernel in the stream is complete
   if (tid == 0 && before_scoring) tc::grid_dep_launch_dependents();
   const uint32_t tmem = X.tmem_slot;
+  // H (fp32 [D][d]) goes through registers into its bf16 operand image H^T (K-major: row c, 64 j per 128-byte row,
+  // two j blocks): thread x of the 16 softmax warps gathers, for DPL items (column c, 8 consecutive j), the eight
+  // values H[j][c]; lanes = consecutive columns, so every load of a warp is one 128-byte line
+  float pre_h[DPL][8];
+  if (tid < 512) {
+    const float* Hg = L.H + (size_t)unit * D * d;
+#pragma unroll
+    for (int n = 0; n < DPL; ++n) {
+      const int it = tid + 512 * n, cc = it % d, jc = it / d;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) pre_h[n][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+    }
+  }
   if (tid < D) X.s_vec[tid] = L.s[(size_t)unit * D + tid];
   __syncthreads();
+  if (tid < 512) {
+#pragma unroll
+    for (int n = 0; n < DPL; ++n) {
+      const int it = tid + 512 * n, cc = it % d, jc = it / d;
+      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(pre_h[n]);
+    }
+    tc::fence_async_smem();
+    tc::mbar_arrive(BAR(A2_HFULL));
+  }
 
   // block `blk` of the key stream -> TMA source
   auto issue_block = [&](uint32_t dst, int blk, bool is_v, uint32_t bar) {
@@ -128,8 +150,6 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   if (warp == 17) {
     // =============================== TMA producer ===============================
     if (lane == 0) {
-      tc::mbar_expect_tx(BAR(A2_HFULL), 2u * d * 128u);
-      tc::bulk_copy_g2s(sbase + S::ht, ht_image + (size_t)unit * (2 * d * 64), 2u * d * 128u, BAR(A2_HFULL));
       // queries: tile w, head slot hs -> rows hs * 64 .. hs * 64 + 63
       tc::mbar_expect_tx(BAR(A2_QFULL), (uint32_t)nw * kblk * 16384u);
       for (int w = 0; w < nw; ++w)

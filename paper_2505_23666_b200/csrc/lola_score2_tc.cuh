@@ -47,7 +47,7 @@ template <int DPL>
 __global__ void __launch_bounds__(kSc2Threads, 1)
 k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __grid_constant__ CUtensorMap tm_gv,
             const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv, const uint4* wt_image,
-            const __nv_bfloat16* ht_image, int tiles_per_cta, int beside_attention) {
+            int tiles_per_cta, int beside_attention) {
   using S = Score2Smem<DPL>;
   if (state_failed(L)) return;                        // an earlier kernel failed: do nothing
   constexpr int d = DPL * 32;
@@ -98,16 +98,18 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
     decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile0 + wg, nGB, nRB, unit, bar_k);
     decode_issue_tile<DPL>(stage + S::st_v, &tm_gv, &tm_wv, tile0 + wg, nGB, nRB, unit, bar_v);
   }
-  // ---- operands: H^T operand image (bulk copies, one per j block), the two parts of s as rows d, d+1,
-  //      W^T image
-  const uint32_t bar_h = sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 48u;
-  if (tid == 0) {
-    tc::mbar_expect_tx(bar_h, 2u * d * 128u);
-    const uint8_t* src = reinterpret_cast<const uint8_t*>(ht_image + (size_t)unit * (2 * d * 64));
-    tc::bulk_copy_g2s(sbase + S::ht, src, d * 128u, bar_h);
-    tc::bulk_copy_g2s(sbase + S::ht + S::ht_blk, src + d * 128, d * 128u, bar_h);
-  }
+  // ---- operands: H^T operand image (from H through registers: thread x gathers, for DPL items (column c, 8
+  //      consecutive j), the eight values H[j][c]; lanes = consecutive columns, so every load of a warp is one
+  //      128-byte line), the two parts of s as rows d, d+1, W^T image
   {
+    float pre_h[DPL][8];
+    const float* Hg = L.H + (size_t)unit * D * d;
+#pragma unroll
+    for (int n = 0; n < DPL; ++n) {
+      const int it = tid + kSc2Threads * n, cc = it % d, jc = it / d;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) pre_h[n][jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
+    }
     const uint4* img = wt_image + (size_t)h * kblk * 512;
     for (int i = tid; i < kblk * 512; i += kSc2Threads)
       *reinterpret_cast<uint4*>(sm + S::b1 + i * 16) = img[i];
@@ -123,8 +125,12 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       const int jb = i / (14 * 8), r = (i / 8) % 14, ch = i % 8;
       *reinterpret_cast<uint4*>(sm + S::ht + jb * S::ht_blk + tc::sw128_off(d + 2 + r, ch)) = make_uint4(0, 0, 0, 0);
     }
+#pragma unroll
+    for (int n = 0; n < DPL; ++n) {
+      const int it = tid + kSc2Threads * n, cc = it % d, jc = it / d;
+      *reinterpret_cast<uint4*>(sm + S::ht + (jc >> 3) * S::ht_blk + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(pre_h[n]);
+    }
   }
-  ok = tc::mbar_wait(bar_h, 0) && ok;
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();

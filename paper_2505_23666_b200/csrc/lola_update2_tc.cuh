@@ -114,8 +114,9 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
       for (int q = 0; q < kblk; ++q) pre_w[q] = img[tid + q * kUp2Threads];
     }
   }
-  // H of the unit streams into shared memory (asynchronous 16-byte copies) meanwhile
-  if (PHASE != 1 && fold) {
+  // H of the unit streams into shared memory (asynchronous 16-byte copies) meanwhile.  PHASE 2 never reads H:
+  // it adds the fold's product to H in memory (reductions at the L2) and keeps no operand image
+  if (PHASE == 0 && fold) {
     const float* Hg = L.H + (size_t)unit * D * d;
     for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
       const int row = i / (d / 4), c4 = i % (d / 4);
@@ -288,19 +289,38 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
     if (tid < nMove) { X.mover[tid] = pre_src; X.free_slot[tid] = pre_dst; }
     __syncthreads();
   }
-  // ---- leaving pairs that stay: into the freed slots, then into the slots beyond count_g
+  // ---- leaving pairs that stay: into the freed slots, then into the slots beyond count_g.  Copies go in
+  // batches of kCopyBatch 16-byte pieces per thread, all loads of a batch before its stores: one round trip to
+  // memory per batch instead of one per piece
+  constexpr int kCopyBatch = 8;
   auto do_movers = [&](int t0, int nt) {
-    for (int i = t0; i < nMove * nch * 2; i += nt) {
-      const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
-      const int src = X.mover[w];
-      const int dst = w < nGL ? X.free_slot[w] : cg + (w - nGL);
-      const T *kp, *vp;
-      locate_leaving<T>(L, c, unit, b, h, c.r_pos0 + src, kp, vp);
-      T* dp = (isv ? (T*)L.gv : (T*)L.gk) + ((size_t)unit * lam + dst) * d;
-      *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
-      if (rem == 0) {
-        L.gpos[(size_t)unit * lam + dst] = c.r_pos0 + src;
-        scu[dst] = fold ? scu[lam + src] : CUDART_NAN_F;             // never scored while the cache still has room
+    const int total = nMove * nch * 2;
+    for (int base = t0; base < total; base += nt * kCopyBatch) {
+      uint4 tmp[kCopyBatch];
+#pragma unroll
+      for (int k = 0; k < kCopyBatch; ++k) {
+        const int i = base + k * nt;
+        if (i < total) {
+          const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+          const T *kp, *vp;
+          locate_leaving<T>(L, c, unit, b, h, c.r_pos0 + X.mover[w], kp, vp);
+          tmp[k] = *reinterpret_cast<const uint4*>((isv ? vp : kp) + ch * 8);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kCopyBatch; ++k) {
+        const int i = base + k * nt;
+        if (i < total) {
+          const int w = i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+          const int src = X.mover[w];
+          const int dst = w < nGL ? X.free_slot[w] : cg + (w - nGL);
+          T* dp = (isv ? (T*)L.gv : (T*)L.gk) + ((size_t)unit * lam + dst) * d;
+          *reinterpret_cast<uint4*>(dp + ch * 8) = tmp[k];
+          if (rem == 0) {
+            L.gpos[(size_t)unit * lam + dst] = c.r_pos0 + src;
+            scu[dst] = fold ? scu[lam + src] : CUDART_NAN_F;         // never scored while the cache still has room
+          }
+        }
       }
     }
   };
@@ -308,12 +328,28 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   auto do_roll = [&](int t0, int nt) {
     if (eta <= 0) return;
     const int first = max(0, c.n - eta);
-    for (int i = t0; i < (c.n - first) * nch * 2; i += nt) {
-      const int ci = first + i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
-      const int p = c.n_seen + ci;
-      const T* sp = (isv ? (const T*)c.v : (const T*)c.k) + (((size_t)b * c.n + ci) * L.Hkv + h) * d;
-      T* dp = (isv ? (T*)L.wv : (T*)L.wk) + ((size_t)unit * eta + (p % eta)) * d;
-      *reinterpret_cast<uint4*>(dp + ch * 8) = *reinterpret_cast<const uint4*>(sp + ch * 8);
+    const int total = (c.n - first) * nch * 2;
+    for (int base = t0; base < total; base += nt * kCopyBatch) {
+      uint4 tmp[kCopyBatch];
+#pragma unroll
+      for (int k = 0; k < kCopyBatch; ++k) {
+        const int i = base + k * nt;
+        if (i < total) {
+          const int ci = first + i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+          const T* sp = (isv ? (const T*)c.v : (const T*)c.k) + (((size_t)b * c.n + ci) * L.Hkv + h) * d;
+          tmp[k] = *reinterpret_cast<const uint4*>(sp + ch * 8);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kCopyBatch; ++k) {
+        const int i = base + k * nt;
+        if (i < total) {
+          const int ci = first + i / (2 * nch), rem = i % (2 * nch), isv = rem / nch, ch = rem % nch;
+          const int p = c.n_seen + ci;
+          T* dp = (isv ? (T*)L.wv : (T*)L.wk) + ((size_t)unit * eta + (p % eta)) * d;
+          *reinterpret_cast<uint4*>(dp + ch * 8) = tmp[k];
+        }
+      }
     }
   };
   if (fold) {
@@ -389,6 +425,35 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
   if (tid >= 256) do_roll(tid - 256, kUp2Threads - 256);             // the movers' reads of the ring ended at the barrier above
   else { ok = tc::mbar_wait(bar, ph) && ok; ph ^= 1; }
   tc::fence_after_sync();
+  if (PHASE == 2) {
+    if (tid < 256 && ok) {                                           // row j = t, columns [hf * d/2, +d/2)
+      // dH from tensor memory into the (padded) rows of the staging area
+      constexpr int HC = d / 2;
+      float* Hrow = reinterpret_cast<float*>(sm + S::hs + (size_t)t * S::hs_row) + hf * HC;
+#pragma unroll
+      for (int c0 = 0; c0 < HC; c0 += 32) {
+        float p[32];
+        tc::tmem_ld32(tm_d + lane_addr + hf * HC + c0, p);
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<float4*>(Hrow + c0 + q * 4) = make_float4(p[q * 4], p[q * 4 + 1], p[q * 4 + 2], p[q * 4 + 3]);
+      }
+      if (hf == 0) {
+        float ds[2];
+        tc::tmem_ld2(tm_d + lane_addr + d, ds);
+        L.s[(size_t)unit * D + t] += ds[0];
+      }
+    }
+    __syncthreads();
+    if (ok) {
+      // H += dH: 16-byte reductions performed at the L2, a warp covers 512 consecutive bytes (nothing is read back)
+      float4* Hg4 = reinterpret_cast<float4*>(L.H + (size_t)unit * D * d);
+      for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
+        const int row = i / (d / 4), c4 = i % (d / 4);
+        atomicAdd(Hg4 + i, *reinterpret_cast<const float4*>(sm + S::hs + (size_t)row * S::hs_row + (size_t)c4 * 16));
+      }
+    }
+  } else {
   if (tid < 256 && ok) {                                             // row j = t, columns [hf * d/2, +d/2)
     // H += dH in the shared-memory copy (this thread owns the half row) and the same values as bf16 in
     // the operand image layout [2 j blocks][d rows c][64 j] (row c, K index j, 128-byte swizzle), staged
@@ -430,6 +495,7 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
     uint4* img4 = reinterpret_cast<uint4*>(ht_image + (size_t)unit * (2 * d * 64));
     for (int i = tid; i < 2 * d * 128 / 16; i += kUp2Threads) img4[i] = *reinterpret_cast<const uint4*>(sm + S::kt + (size_t)i * 16);
   }
+  }  // (PHASE 0: H and its image through shared memory)
   }  // fold
   if (!fold) {
     do_movers(tid, kUp2Threads);
@@ -452,23 +518,6 @@ __global__ void __launch_bounds__(kUp2Threads, 1) k_update2_tc(Layer L, Call c, 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   update2_body<DPL, PHASE>(L, c, wt_image, ht_image, sm, (int)blockIdx.x);
-}
-
-// Rebuilds the bf16 operand image of H for every unit (after a path that changed H without
-// maintaining it): per unit [2 j blocks][d rows c][64 j], 128-byte swizzle.
-template <int DPL>
-__global__ void __launch_bounds__(256) k_build_ht_image(Layer L, __nv_bfloat16* ht_image) {
-  constexpr int d = DPL * 32, D = 128;
-  const int unit = blockIdx.x;
-  const float* Hg = L.H + (size_t)unit * D * d;
-  uint8_t* img = reinterpret_cast<uint8_t*>(ht_image + (size_t)unit * (2 * d * 64));
-  for (int i = threadIdx.x; i < d * (D / 8); i += 256) {
-    const int cc = i % d, jc = i / d;
-    float f8[8];
-#pragma unroll
-    for (int jj = 0; jj < 8; ++jj) f8[jj] = Hg[(size_t)(jc * 8 + jj) * d + cc];
-    *reinterpret_cast<uint4*>(img + (jc >> 3) * (d * 128) + tc::sw128_off(cc, jc & 7)) = tc::pack8_bf16(f8);
-  }
 }
 
 }  // namespace lola
