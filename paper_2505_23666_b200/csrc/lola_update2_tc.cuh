@@ -444,11 +444,12 @@ __device__ __forceinline__ void update2_body(const Layer& L, const Call& c, cons
         L.s[(size_t)unit * D + t] += ds[0];
       }
     }
-    __syncthreads();
-    if (ok) {
+    // (the lower half alone: the upper half is still rolling the window)
+    if (tid < 256) tc::named_bar_sync(2, 256);
+    if (tid < 256 && ok) {
       // H += dH: 16-byte reductions performed at the L2, a warp covers 512 consecutive bytes (nothing is read back)
       float4* Hg4 = reinterpret_cast<float4*>(L.H + (size_t)unit * D * d);
-      for (int i = tid; i < D * (d / 4); i += kUp2Threads) {
+      for (int i = tid; i < D * (d / 4); i += 256) {
         const int row = i / (d / 4), c4 = i % (d / 4);
         atomicAdd(Hg4 + i, *reinterpret_cast<const float4*>(sm + S::hs + (size_t)row * S::hs_row + (size_t)c4 * 16));
       }
