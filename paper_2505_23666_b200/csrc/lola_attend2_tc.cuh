@@ -267,6 +267,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     const uint32_t tm_sb = tm_s + (uint32_t)hf * 64u;  // this thread's 64 score columns; its weights go to the first 32
     const uint32_t tm_o = tmem + 256u + (uint32_t)w * 128u + lane_addr;
     constexpr int HC = d / 2;
+    const int pair_bar = 1 + w * 4 + wq;               // the two warps that share this row quadrant (64 threads)
     // ---- linear term first
     ok = WAIT(A2_SFULL + w, 0) && ok;                  // U = Q W is in the first 64 score columns
     tc::fence_after_sync();
@@ -349,7 +350,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
       }
       X.hx[w][hf][t] = fmaxf(mx0, mx1);
-      tc::named_bar_sync(1 + w, 256);                  // (also: both halves hold their scores in registers now)
+      tc::named_bar_sync(pair_bar, 64);                    // (also: both halves hold their scores in registers now)
       const float m_tile = fmaxf(X.hx[w][0][t], X.hx[w][1][t]) * sl2;
       const bool grow = m_tile > m_used + kGrow;
       if (__any_sync(0xffffffffu, grow)) {             // rare; tensor-memory accesses are warp-wide: every lane takes part
@@ -401,9 +402,9 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
     }
     // ---- the two halves of the row's denominator meet (the extra barrier: the partner has read this row's last
     // maxima before the slot is reused)
-    tc::named_bar_sync(1 + w, 256);
+    tc::named_bar_sync(pair_bar, 64);  
     X.hx[w][hf][t] = l;
-    tc::named_bar_sync(1 + w, 256);
+    tc::named_bar_sync(pair_bar, 64);  
     const float lden = X.hx[w][hf ^ 1][t];
     ok = WAIT(A2_ODONE + w, NT & 1) && ok;
     tc::fence_after_sync();
@@ -432,7 +433,7 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
         }
       }
       tc::fence_async_smem();
-      tc::named_bar_sync(1 + w, 256);
+      tc::named_bar_sync(9 + w, 256);
       if (t == 0 && hf == 0 && ok) {
         const uint32_t sstg = sbase + stg_off;
         for (int s2 = 0; s2 < 2; ++s2) {
