@@ -20,7 +20,10 @@
  *     kernels are chained by programmatic dependent launches on that one stream), and the fold follows both.
  *   - Work is enqueued on the given stream (a cudaStream_t passed as void*; NULL = legacy default
  *     stream) and the call returns without synchronising unless stated otherwise.  All calls on
- *     one state must be issued on one stream, or be ordered by the caller.
+ *     one state must be issued on one stream, or be ordered by the caller.  The kernels of a call are
+ *     launched with programmatic stream serialization and read the call's q before they wait for the
+ *     work ahead of them in the stream: what writes q, k, v must be complete in the ordinary way (a
+ *     copy, or a kernel that does not signal programmatic launch completion before its end).
  *   - Return value: LOLA_OK (0) or a negative error code.  Argument errors are found on the host
  *     before anything is enqueued and leave the state untouched.  Nothing throws, prints or exits.
  *   - One state serves `batch` sequences that advance in lock-step (equal lengths, no padding).

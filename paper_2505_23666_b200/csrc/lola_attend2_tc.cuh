@@ -107,6 +107,22 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
+  if (warp == 17 && lane == 0) {
+    // The queries are an input of the call, not something the kernels before this one in the stream produce (those
+    // are this library's own, which write the memories and outputs only, or kernels that let nothing start before
+    // they are complete): their load starts before the wait, so that U = Q W can begin as soon as W^T arrives.
+    // queries: tile w, head slot hs -> rows hs * 64 .. hs * 64 + 63
+    tc::mbar_expect_tx(BAR(A2_QFULL), (uint32_t)nw * kblk * 16384u);
+    for (int w = 0; w < nw; ++w)
+      for (int hs = 0; hs < 2; ++hs) {
+        const int hl = (qt0 + w) * 2 + hs;
+        const int head = hl < g ? h * g + hl : L.Hq;        // a head index outside the tensor reads as zeros
+#pragma unroll
+        for (int cb = 0; cb < kblk; ++cb)
+          tc::tma_load_4d(sbase + S::q + (uint32_t)w * 32768u + (uint32_t)cb * 16384u + (uint32_t)hs * 8192u, &tm_q, cb * 64, head,
+                          0, b, BAR(A2_QFULL));
+      }
+  }
   tc::grid_dep_wait();                               // everything before this kernel in the stream is complete
   if (tid == 0 && before_scoring) tc::grid_dep_launch_dependents();
   const uint32_t tmem = X.tmem_slot;
@@ -150,17 +166,6 @@ k_attend2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
   if (warp == 17) {
     // =============================== TMA producer ===============================
     if (lane == 0) {
-      // queries: tile w, head slot hs -> rows hs * 64 .. hs * 64 + 63
-      tc::mbar_expect_tx(BAR(A2_QFULL), (uint32_t)nw * kblk * 16384u);
-      for (int w = 0; w < nw; ++w)
-        for (int hs = 0; hs < 2; ++hs) {
-          const int hl = (qt0 + w) * 2 + hs;
-          const int head = hl < g ? h * g + hl : L.Hq;          // a head index outside the tensor reads as zeros
-#pragma unroll
-          for (int cb = 0; cb < kblk; ++cb)
-            tc::tma_load_4d(sbase + S::q + (uint32_t)w * 32768u + (uint32_t)cb * 16384u + (uint32_t)hs * 8192u, &tm_q, cb * 64, head,
-                            0, b, BAR(A2_QFULL));
-        }
       // W^T image into the key buffer of stage 1, which the second tile takes over once U = Q W has read it
       tc::mbar_expect_tx(BAR(A2_WFULL), (uint32_t)kblk * 8192u);
       tc::bulk_copy_g2s(sbase + S::stage0 + S::stage_bytes + S::st_k, wt_image + (size_t)h * kblk * 512, kblk * 8192u, BAR(A2_WFULL));
