@@ -77,13 +77,14 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
 
   const uint32_t bar_k = sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + (uint32_t)wg * 24u;
   const uint32_t bar_v = bar_k + 8, bar_mma = bar_k + 16;
+  const uint32_t bar_u = sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 48u + (uint32_t)wg * 8u;
   const uint32_t stage = sbase + S::stage0 + (uint32_t)wg * S::stage_bytes;
   uint8_t* stage_p = sm + S::stage0 + (size_t)wg * S::stage_bytes;
-  uint32_t pk = 0, pv = 0, pm = 0;
+  uint32_t pk = 0, pv = 0, pm = 0, pu = 0;
   bool ok = true;
 
   if (tid == 0) {
-    for (int i = 0; i < 7; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 8u * i, 1);
+    for (int i = 0; i < 8; ++i) tc::mbar_init(sbase + S::misc + (uint32_t)offsetof(Score2Misc, bars) + 8u * i, 1);
     tc::mbar_init_fence();
   }
   if (warp == 0) tc::tmem_alloc(&X.tmem_slot, 512);
@@ -137,14 +138,26 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
   tc::fence_after_sync();
   const uint32_t tmem = X.tmem_slot;
   const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-  const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // U, then [P | den]
-  const uint32_t tm_phi = tm_a + 192u;
+  const uint32_t tm_a = tmem + (uint32_t)wg * 256u;            // [P | den]
+  const uint32_t tm_phi = tm_a + 192u;                         // U = K W of a tile, then its feature map in place (bf16 pairs)
   const uint32_t idesc1 = tc::make_idesc_bf16(128, 64, false, false);
   const uint32_t idesc2 = tc::make_idesc_bf16(128, d + 16, false, false);
   // operand descriptors once; a K step adds its byte offset / 16 to the address field
   const uint64_t dk = tc::make_desc_sw128(stage + S::st_k, 16, 1024), db1 = tc::make_desc_sw128(sbase + S::b1, 16, 1024),
                  dht = tc::make_desc_sw128(sbase + S::ht, 16, 1024);
 
+  // U = K W of a tile is issued one tile ahead: right behind [P | den] of the tile before (the tensor pipe runs
+  // in order, so the feature map there is consumed first), and runs while the row group works on Eq. 10
+  auto issue_u = [&]() {
+    ok = tc::mbar_wait(bar_k, pk) && ok; pk ^= 1;
+    tc::fence_after_sync();
+#pragma unroll
+    for (int ks = 0; ks < d / 16; ++ks)
+      tc::mma_bf16_ss(tm_phi, dk + (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
+                      db1 + (uint64_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), idesc1, ks > 0);
+    tc::mma_commit(bar_u);
+  };
+  if (lead && tile0 + wg < tile1) issue_u();
   if (wg == 1) asm volatile("bar.arrive 3, 512;" ::: "memory");   // row group 0 takes the first turn
 
   for (int tile = tile0 + wg; tile < tile1; tile += 2) {
@@ -161,23 +174,16 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       if (off < cw && p < c.r_pos0 + c.r && p >= c.r_pos0) e_idx = lam + (p - c.r_pos0);
     }
 
-    ok = tc::mbar_wait(bar_k, pk) && ok; pk ^= 1;
-    tc::fence_after_sync();
-    if (lead) {
-#pragma unroll
-      for (int ks = 0; ks < d / 16; ++ks)
-        tc::mma_bf16_ss(tm_a, dk + (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4),
-                        db1 + (uint64_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), idesc1, ks > 0);
-      tc::mma_commit(bar_mma);
-    }
-    ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
+    ok = tc::mbar_wait(bar_u, pu) && ok; pu ^= 1;     // U of this tile is complete (and the key tile is read)
     tc::fence_after_sync();
     if (lead && tile + 2 < tile1) decode_issue_tile<DPL>(stage + S::st_k, &tm_gk, &tm_wk, tile + 2, nGB, nRB, unit, bar_k);
     {
       tc::named_bar_sync(3 + wg, 512);
       uint32_t u[64], pk2[32];
-      tc::tmem_ld64u(tm_a + lane_addr, u);
+      tc::tmem_ld64u(tm_phi + lane_addr, u);
       tc::phi_half(u, hf != 0, L.phi_kind == 1, pk2);
+      tc::fence_before_sync();
+      tc::named_bar_sync(1 + wg, 256);               // both threads of a row have read U: its columns take the feature map
       tc::tmem_st32u(tm_phi + lane_addr + hf * 32, pk2);
       if (wg == 0) asm volatile("bar.arrive 4, 512;" ::: "memory"); else asm volatile("bar.arrive 3, 512;" ::: "memory");
     }
@@ -189,6 +195,7 @@ k_score2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const __
       for (int ks = 0; ks < D / 16; ++ks)
         tc::mma_bf16_ts(tm_a, tm_phi + ks * 8, dht + (uint64_t)(((ks >> 2) * S::ht_blk + (ks & 3) * 32) >> 4), idesc2, ks > 0);
       tc::mma_commit(bar_mma);
+      if (tile + 2 < tile1) issue_u();               // U of this row group's next tile
     }
     ok = tc::mbar_wait(bar_v, pv) && ok; pv ^= 1;
     ok = tc::mbar_wait(bar_mma, pm) && ok; pm ^= 1;
