@@ -359,25 +359,22 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       const bool valid = R < lam || R - lam < eta;
       ok = tc::mbar_wait(bar_u(i), (uint32_t)(tile >> 1) & 1u, abw) && ok;
       tc::fence_after_sync();
-      // q.k of this row (log2 units) and the warp's maxima: the score group turns them into weights
+      // [U | Z] of this row in one round trip to tensor memory: this thread's q.k columns (log2 units after
+      // scaling; their warp maxima go to the score group, which turns them into weights) and all of U
       float z[QH], wm[QH];
-      {
-        float zraw[QH];
-        if (QH == 4) tc::tmem_ld4(tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<float(&)[4]>(zraw));
-        else tc::tmem_ld2(tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<float(&)[2]>(zraw));
-#pragma unroll
-        for (int r = 0; r < QH; ++r) {
-          z[r] = valid ? zraw[r] * sl2 : -CUDART_INF_F;
-          wm[r] = warp_max_redux(z[r]);
-        }
-      }
-      // this thread's half of the feature map: hf = 0: softmax(u), hf = 1: softmax(-u)
       uint32_t pk2[32];
       {
-        uint32_t u[64];
-        tc::tmem_ld64u(tm_uz(i) + lane_addr, u);
+        uint32_t u[64], zraw[QH];
+        if (QH == 4) tc::tmem_ld64u_and4(tm_uz(i) + lane_addr, u, tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<uint32_t(&)[4]>(zraw));
+        else tc::tmem_ld64u_and2(tm_uz(i) + lane_addr, u, tm_uz(i) + lane_addr + 64 + hf * QH, reinterpret_cast<uint32_t(&)[2]>(zraw));
         tc::fence_before_sync();
         tc::mbar_arrive(bar_uread(i));               // [U | Z] of this tile is in registers: the buffer may take tile + 2
+#pragma unroll
+        for (int r = 0; r < QH; ++r) {
+          z[r] = valid ? __uint_as_float(zraw[r]) * sl2 : -CUDART_INF_F;
+          wm[r] = warp_max_redux(z[r]);
+        }
+        // this thread's half of the feature map: hf = 0: softmax(u), hf = 1: softmax(-u)
         tc::phi_half(u, hf != 0, exp_kind, pk2);
       }
       if (tile >= 2) {                               // the score group is done with the buffers of tile - 2
@@ -525,17 +522,21 @@ k_decode2_tc(Layer L, Call c, const __grid_constant__ CUtensorMap tm_gk, const _
       // ---- Eq. 10: this thread's half of the value columns
       float ss;
       {
-        float dn[2];
-        tc::tmem_ld2(tm_p + lane_addr + d, dn);
-        const float den = dn[0] + dn[1];
-        const float inv = den > 0.f ? 1.0f / den : 0.f;
         // packed pairs: d = v - P / den, four running sums of squares (columns 4k, 4k+1 | 4k+2, 4k+3)
-        const uint64_t ninv2 = tc::pack_f2(-inv, -inv);
+        uint64_t ninv2 = 0;
         uint64_t accA = tc::pack_f2(0.f, 0.f), accB = accA;
 #pragma unroll
         for (int c0 = 0; c0 < HC; c0 += 32) {
           uint32_t p[32];
-          tc::tmem_ld32u(tm_p + lane_addr + hf * HC + c0, p);
+          if (c0 == 0) {                                 // the two parts of the denominator come with the first columns
+            uint32_t dn[2];
+            tc::tmem_ld32u_and2(tm_p + lane_addr + hf * HC, p, tm_p + lane_addr + d, dn);
+            const float den = __uint_as_float(dn[0]) + __uint_as_float(dn[1]);
+            const float inv = den > 0.f ? 1.0f / den : 0.f;
+            ninv2 = tc::pack_f2(-inv, -inv);
+          } else {
+            tc::tmem_ld32u(tm_p + lane_addr + hf * HC + c0, p);
+          }
           if (c0 + 32 >= HC) {                 // [P | den] is read: the next tile's product may overwrite it
             tc::fence_before_sync();
             tc::mbar_arrive(bar_pfree);
